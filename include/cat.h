@@ -1,0 +1,203 @@
+/*
+ * cat.h -- C ABI of the B200 (sm_100a) CAT library.
+ *
+ * CAT (Cluster-based Affine Transformation) corrects the outputs of a low-bit
+ * quantised (LQ) model towards those of its full-precision (FP) counterpart:
+ * the LQ output rows are clustered with K-Means, each cluster k gets an
+ * element-wise affine map (gamma_k, beta_k) fitted in closed form against the
+ * FP outputs, and at inference a row is assigned to its nearest centroid and
+ * corrected with that cluster's map.
+ *
+ * Conventions for every entry point unless stated otherwise
+ *   - All data pointers are DEVICE pointers owned by the caller; matrices are
+ *     fp32, row-major, contiguous (leading dimension D); base addresses must
+ *     be 16-byte aligned.  Labels are 0-based int32.
+ *   - `workspace` is caller-provided device scratch of at least the size the
+ *     matching *_workspace_bytes query returns (256-byte aligned).  The
+ *     library allocates and frees nothing.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls only enqueue work: they return after launching, never synchronise,
+ *     and are re-entrant for distinct workspaces.
+ *   - Return value: CAT_OK or an error code; on error nothing was enqueued
+ *     (argument errors) or outputs are undefined (CAT_ERR_CUDA).  The library
+ *     never throws, aborts or traps.
+ *   - Inputs must be finite.  Non-finite values give unspecified labels but
+ *     never an out-of-range label or an invalid memory access.
+ *   - Limits: 1 <= K <= CAT_MAX_K, K <= N < 2^31, 1 <= D <= CAT_MAX_D.
+ *     D % 4 != 0 is supported through scalar loads (slower).
+ */
+#ifndef CAT_H_
+#define CAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int cat_status_t;
+
+enum {
+    CAT_OK = 0,
+    CAT_ERR_NULL = 1,        /* a required pointer is NULL */
+    CAT_ERR_SHAPE = 2,       /* N < K, K < 1, D < 1, iters < 0, alpha outside [0,1] */
+    CAT_ERR_ALIGN = 3,       /* a base pointer is not 16-byte aligned */
+    CAT_ERR_WORKSPACE = 4,   /* workspace NULL or smaller than the query says */
+    CAT_ERR_CUDA = 5,        /* a CUDA runtime call failed: see cat_last_cuda_error() */
+    CAT_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait gave up (reported by cat_device_status) */
+    CAT_ERR_UNSUPPORTED = 7  /* K > CAT_MAX_K, D > CAT_MAX_D or N >= 2^31 */
+};
+
+#define CAT_MAX_K 512
+#define CAT_MAX_D 16384
+
+/* Diagnostics of one cat_fit call, written to device memory (all int64). */
+typedef struct cat_fit_diag {
+    int64_t refined_rows_total;   /* rows whose label needed the exact fp64 pass, summed over all assignments */
+    int64_t refined_rows_final;   /* same, final assignment only */
+    int64_t empty_clusters_final; /* clusters with no rows in the final assignment */
+    int64_t device_status;        /* CAT_OK or CAT_ERR_DEVICE_TIMEOUT */
+} cat_fit_diag_t;
+
+/* ---- the two calls of the hot path ------------------------------------ */
+
+/*
+ * CAT fitting (Algorithm 1 "CAT Fitting" with the cluster model fitted on the
+ * rows themselves; Section 3.1 for the closed form; Section 4 Setup: K-Means).
+ *
+ *   1. centroids <- init_centroids, or the first K rows of Yq when NULL
+ *   2. `iters` Lloyd rounds: label_i = argmin_k ||Yq_i - c_k||^2 (lowest k on
+ *      ties); c_k <- mean of its rows (a cluster with no rows keeps c_k)
+ *   3. final assignment against the final centroids -> labels_out
+ *   4. per cluster k and column j over the rows of the cluster:
+ *        muQ, muF = means of Yq, Yfp;  var = mean (q-muQ)^2;  cov = mean (q-muQ)(f-muF)
+ *        gamma = cov / max(var, 1e-8);  beta = muF - gamma*muQ
+ *      empty cluster: gamma = 1, beta = 0.
+ *
+ * Yq, Yfp       [N, D] in.   centroids_out, gamma_out, beta_out  [K, D] out.
+ * labels_out    [N] out, may be NULL.
+ * init_centroids [K, D] in, may be NULL; must not alias centroids_out.
+ * diag          device pointer to one cat_fit_diag_t, may be NULL.
+ * Labels are decided in fp64 whenever the fast fp32 scores cannot separate
+ * the two nearest centroids; sums and moments are accumulated in fp64.
+ */
+size_t cat_fit_workspace_bytes(int64_t N, int32_t D, int32_t K);
+
+cat_status_t cat_fit(const float *Yq, const float *Yfp, int64_t N, int32_t D, int32_t K,
+                     int32_t iters, float *centroids_out, float *gamma_out, float *beta_out,
+                     int32_t *labels_out, void *workspace, size_t workspace_bytes, void *stream);
+
+cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t D, int32_t K,
+                          int32_t iters, const float *init_centroids,
+                          float *centroids_out, float *gamma_out, float *beta_out,
+                          int32_t *labels_out, cat_fit_diag_t *diag,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * CAT inference (Algorithm 2 "CAT Inferencing" without PCA, alpha = 1):
+ *   label_i = argmin_k ||Yq_i - c_k||^2 ;  Y_out_i = gamma_label * Yq_i + beta_label
+ * evaluated as one fused multiply-add per element (a single rounding).
+ *
+ * Yq [N, D] in; centroids, gamma, beta [K, D] in; Y_out [N, D] out (must not
+ * overlap Yq); labels_out [N] out, may be NULL.  N >= 1 (N < K is allowed).
+ */
+size_t cat_apply_workspace_bytes(int64_t N, int32_t D, int32_t K);
+
+cat_status_t cat_apply(const float *Yq, int64_t N, int32_t D, int32_t K,
+                       const float *centroids, const float *gamma, const float *beta,
+                       float *Y_out, int32_t *labels_out,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The alpha-blended correction of Section 3.1 / Algorithm 2:
+ *   Y_out_i = Yq_i + alpha * ((gamma_l * Yq_i + beta_l) - Yq_i),  0 <= alpha <= 1.
+ * Evaluated as fma(1 + alpha*(gamma-1), y, alpha*beta) with the two
+ * coefficients formed in fp64 per element.  alpha = 1 is exactly cat_apply.
+ */
+cat_status_t cat_apply_blend(const float *Yq, int64_t N, int32_t D, int32_t K,
+                             const float *centroids, const float *gamma, const float *beta,
+                             float alpha, float *Y_out, int32_t *labels_out,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- step-level entry points (the same kernels cat_fit chains; used for
+ *      row-sharded multi-GPU fitting and for step-wise checks) ------------ */
+
+/* Nearest-centroid labels only (the cluster model's "predict", Alg. 2 step 2).
+ * Workspace: cat_apply_workspace_bytes(N, D, K). */
+cat_status_t cat_assign(const float *Yq, int64_t N, int32_t D, int32_t K,
+                        const float *centroids, int32_t *labels_out,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/* Per-cluster column sums of Y (fp64) and cluster sizes for given labels:
+ * sums_out [K, D] double, counts_out [K] int64.  Labels must lie in [0, K).
+ * Rows are added in a fixed order: results are reproducible run to run.
+ * Workspace: cat_fit_workspace_bytes(N, D, K). */
+cat_status_t cat_cluster_sums(const float *Y, const int32_t *labels, int64_t N, int32_t D,
+                              int32_t K, double *sums_out, int64_t *counts_out,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/* c_k <- float(sums_k / counts_k) where counts_k > 0, else unchanged. */
+cat_status_t cat_centroids_from_sums(const double *sums, const int64_t *counts, int32_t D,
+                                     int32_t K, float *centroids_inout, void *stream);
+
+/* Centred second moments for given labels and cluster means (fp64):
+ *   var_out[k,j] = sum_{i in k} (q_ij - meanQ[k,j])^2
+ *   cov_out[k,j] = sum_{i in k} (q_ij - meanQ[k,j]) (f_ij - meanF[k,j])
+ * (sums, not yet divided by the cluster size).  Workspace as for cat_fit. */
+cat_status_t cat_centred_moments(const float *Yq, const float *Yfp, const int32_t *labels,
+                                 int64_t N, int32_t D, int32_t K,
+                                 const double *meanQ, const double *meanF,
+                                 double *var_out, double *cov_out,
+                                 void *workspace, size_t workspace_bytes, void *stream);
+
+/* gamma/beta from cluster sums and centred moment sums (Algorithm 1 steps
+ * after the means): n = counts[k]; n == 0 -> (1, 0); else
+ * gamma = (cov/n) / max(var/n, 1e-8), beta = sumF/n - gamma*sumQ/n. */
+cat_status_t cat_solve_gamma_beta(const double *sumQ, const double *sumF,
+                                  const double *var_sum, const double *cov_sum,
+                                  const int64_t *counts, int32_t D, int32_t K,
+                                  float *gamma_out, float *beta_out, void *stream);
+
+/* ---- host-buffer entry points (end-to-end use) ------------------------- */
+
+/*
+ * cat_apply with HOST inputs and outputs.  Yq_host / Y_out_host [N, D] and
+ * labels_out_host [N] (may be NULL) are host pointers, ideally page-locked so
+ * that copies overlap compute; centroids/gamma/beta [K, D] are host pointers
+ * too.  Rows are streamed through device staging buffers carved from
+ * `workspace` (device memory, size from cat_apply_host_workspace_bytes) in
+ * chunks, overlapping H2D copy, the fused kernel and D2H copy.  The call
+ * BLOCKS until all results are on the host.
+ */
+size_t cat_apply_host_workspace_bytes(int64_t N, int32_t D, int32_t K);
+
+cat_status_t cat_apply_host(const float *Yq_host, int64_t N, int32_t D, int32_t K,
+                            const float *centroids_host, const float *gamma_host,
+                            const float *beta_host, float *Y_out_host, int32_t *labels_out_host,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * cat_fit with HOST inputs and outputs: copies Yq/Yfp to device buffers carved
+ * from `workspace` (size from cat_fit_host_workspace_bytes), runs cat_fit and
+ * copies centroids, gamma, beta and (if not NULL) labels back.  BLOCKS until
+ * done.
+ */
+size_t cat_fit_host_workspace_bytes(int64_t N, int32_t D, int32_t K);
+
+cat_status_t cat_fit_host(const float *Yq_host, const float *Yfp_host, int64_t N, int32_t D,
+                          int32_t K, int32_t iters, float *centroids_out_host,
+                          float *gamma_out_host, float *beta_out_host, int32_t *labels_out_host,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- misc --------------------------------------------------------------- */
+
+const char *cat_status_string(cat_status_t status);
+int cat_last_cuda_error(void);           /* cudaError_t of the last failing runtime call on this thread */
+const char *cat_version(void);
+int64_t cat_kernel_launches(void);       /* kernels launched by this library in this process so far */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAT_H_ */

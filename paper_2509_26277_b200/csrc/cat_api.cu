@@ -1,0 +1,332 @@
+// C ABI of libcat.so: argument checks, workspace carving and the launch sequences of
+// cat_fit / cat_apply and the step-level entry points declared in cat.h.
+#include "cat_internal.cuh"
+
+#include <atomic>
+
+namespace cat {
+
+thread_local int g_last_cuda_error = 0;
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---------------------------------------------------------------- workspace carving
+struct Carver {
+    unsigned char *base;
+    size_t off = 0;
+    explicit Carver(void *b) : base(reinterpret_cast<unsigned char *>(b)) {}
+    template <class T>
+    T *take(size_t count)
+    {
+        off = align_up(off, 256);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += count * sizeof(T);
+        return p;
+    }
+};
+
+static void carve_assign_into(Carver &c, AssignWs &w, int64_t N, int D, int K)
+{
+    w.ctl = c.take<Control>(1);
+    w.cnorm = c.take<float>((size_t)K);
+    w.refine_rows = c.take<int32_t>((size_t)N);
+    w.labels = c.take<int32_t>((size_t)N);
+    w.gamma_b = c.take<float>((size_t)K * D);
+    w.beta_b = c.take<float>((size_t)K * D);
+}
+
+AssignWs carve_assign(void *base, int64_t N, int D, int K)
+{
+    Carver c(base);
+    AssignWs w{};
+    carve_assign_into(c, w, N, D, K);
+    w.bytes = align_up(c.off, 256);
+    return w;
+}
+
+FitWs carve_fit(void *base, int64_t N, int D, int K)
+{
+    Carver c(base);
+    FitWs w{};
+    carve_assign_into(c, w.a, N, D, K);
+    SumGeom g1 = sum_geometry(N, D, K, 1);
+    SumGeom g2 = sum_geometry(N, D, K, 2);
+    int nch = g1.nchunks > g2.nchunks ? g1.nchunks : g2.nchunks;
+    size_t KD = (size_t)K * D;
+    w.partial = c.take<double>((size_t)nch * 2 * KD);
+    w.partial_cnt = c.take<int32_t>((size_t)nch * K);
+    w.sumQ = c.take<double>(KD);
+    w.sumF = c.take<double>(KD);
+    w.var = c.take<double>(KD);
+    w.cov = c.take<double>(KD);
+    w.meanQ = c.take<double>(KD);
+    w.meanF = c.take<double>(KD);
+    w.counts = c.take<int64_t>((size_t)K);
+    w.bytes = align_up(c.off, 256);
+    return w;
+}
+
+// ---------------------------------------------------------------- validation
+static cat_status_t check_shape(int64_t N, int32_t D, int32_t K, bool need_n_ge_k)
+{
+    if (K < 1 || D < 1 || N < 1) return CAT_ERR_SHAPE;
+    if (need_n_ge_k && N < K) return CAT_ERR_SHAPE;
+    if (K > CAT_MAX_K || D > CAT_MAX_D || N >= ((int64_t)1 << 31)) return CAT_ERR_UNSUPPORTED;
+    return CAT_OK;
+}
+
+#define CAT_CUDA(expr)                                  \
+    do {                                                \
+        if (!cuda_ok((expr))) return CAT_ERR_CUDA;      \
+    } while (0)
+
+// norms -> fast assignment -> exact pass for undecided rows
+static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const float *C,
+                               int32_t *labels, const AssignWs &w, const float *gamma,
+                               const float *beta, float *out, cudaStream_t s)
+{
+    CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s));
+    CAT_CUDA(launch_assign(Y, N, D, K, C, w.cnorm, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
+    if (K > 1) CAT_CUDA(launch_refine(Y, N, D, K, C, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
+    return CAT_OK;
+}
+
+// per-cluster column sums of M (+ counts) into sums / counts
+static cat_status_t run_cluster_sums(const float *M, const int32_t *labels, int64_t N, int D, int K,
+                                     const FitWs &w, double *sums, int64_t *counts, cudaStream_t s)
+{
+    SumGeom g = sum_geometry(N, D, K, 1);
+    CAT_CUDA(launch_cluster_partial(M, nullptr, labels, N, D, K, g, nullptr, nullptr, 0, w.partial,
+                                    w.partial_cnt, s));
+    CAT_CUDA(launch_reduce_partials(w.partial, w.partial_cnt, g.nchunks, 2, 0, D, K, sums, counts, s));
+    return CAT_OK;
+}
+
+static cat_status_t run_centred(const float *Yq, const float *Yfp, const int32_t *labels, int64_t N,
+                                int D, int K, const FitWs &w, const double *meanQ,
+                                const double *meanF, double *var, double *cov, cudaStream_t s)
+{
+    SumGeom g = sum_geometry(N, D, K, 2);
+    if (g.nacc == 2) {
+        CAT_CUDA(launch_cluster_partial(Yq, Yfp, labels, N, D, K, g, meanQ, meanF, 3, w.partial,
+                                        w.partial_cnt, s));
+        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 0, D, K, var, nullptr, s));
+        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 1, D, K, cov, nullptr, s));
+    } else {
+        CAT_CUDA(launch_cluster_partial(Yq, Yfp, labels, N, D, K, g, meanQ, meanF, 1, w.partial,
+                                        w.partial_cnt, s));
+        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 0, D, K, var, nullptr, s));
+        CAT_CUDA(launch_cluster_partial(Yq, Yfp, labels, N, D, K, g, meanQ, meanF, 2, w.partial,
+                                        w.partial_cnt, s));
+        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 1, D, K, cov, nullptr, s));
+    }
+    return CAT_OK;
+}
+
+}  // namespace cat
+
+using namespace cat;
+
+extern "C" {
+
+size_t cat_apply_workspace_bytes(int64_t N, int32_t D, int32_t K)
+{
+    if (check_shape(N, D, K, false) != CAT_OK) return 0;
+    return carve_assign(nullptr, N, D, K).bytes;
+}
+
+size_t cat_fit_workspace_bytes(int64_t N, int32_t D, int32_t K)
+{
+    if (check_shape(N, D, K, false) != CAT_OK) return 0;
+    return carve_fit(nullptr, N, D, K).bytes;
+}
+
+cat_status_t cat_apply_blend(const float *Yq, int64_t N, int32_t D, int32_t K,
+                             const float *centroids, const float *gamma, const float *beta,
+                             float alpha, float *Y_out, int32_t *labels_out, void *workspace,
+                             size_t workspace_bytes, void *stream)
+{
+    if (!Yq || !centroids || !gamma || !beta || !Y_out) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (!(alpha >= 0.f && alpha <= 1.f)) return CAT_ERR_SHAPE;
+    if (!aligned16(Yq) || !aligned16(centroids) || !aligned16(gamma) || !aligned16(beta) ||
+        !aligned16(Y_out) || (labels_out && !aligned16(labels_out)))
+        return CAT_ERR_ALIGN;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_apply_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    AssignWs w = carve_assign(workspace, N, D, K);
+    int32_t *labels = labels_out ? labels_out : w.labels;
+    const float *g = gamma, *b = beta;
+    if (alpha != 1.f) {
+        CAT_CUDA(launch_blend_params(gamma, beta, alpha, (int64_t)K * D, w.gamma_b, w.beta_b, s));
+        g = w.gamma_b;
+        b = w.beta_b;
+    }
+    return run_assign(Yq, N, D, K, centroids, labels, w, g, b, Y_out, s);
+}
+
+cat_status_t cat_apply(const float *Yq, int64_t N, int32_t D, int32_t K, const float *centroids,
+                       const float *gamma, const float *beta, float *Y_out, int32_t *labels_out,
+                       void *workspace, size_t workspace_bytes, void *stream)
+{
+    return cat_apply_blend(Yq, N, D, K, centroids, gamma, beta, 1.f, Y_out, labels_out, workspace,
+                           workspace_bytes, stream);
+}
+
+cat_status_t cat_assign(const float *Yq, int64_t N, int32_t D, int32_t K, const float *centroids,
+                        int32_t *labels_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!Yq || !centroids || !labels_out) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (!aligned16(Yq) || !aligned16(centroids) || !aligned16(labels_out)) return CAT_ERR_ALIGN;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_apply_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    AssignWs w = carve_assign(workspace, N, D, K);
+    return run_assign(Yq, N, D, K, centroids, labels_out, w, nullptr, nullptr, nullptr,
+                      reinterpret_cast<cudaStream_t>(stream));
+}
+
+cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t D, int32_t K,
+                          int32_t iters, const float *init_centroids, float *centroids_out,
+                          float *gamma_out, float *beta_out, int32_t *labels_out,
+                          cat_fit_diag_t *diag, void *workspace, size_t workspace_bytes,
+                          void *stream)
+{
+    if (!Yq || !Yfp || !centroids_out || !gamma_out || !beta_out) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, true);
+    if (st != CAT_OK) return st;
+    if (iters < 0) return CAT_ERR_SHAPE;
+    if (!aligned16(Yq) || !aligned16(Yfp) || !aligned16(centroids_out) || !aligned16(gamma_out) ||
+        !aligned16(beta_out) || (labels_out && !aligned16(labels_out)) ||
+        (init_centroids && !aligned16(init_centroids)) || (diag && !aligned16(diag)))
+        return CAT_ERR_ALIGN;
+    if (init_centroids == centroids_out) return CAT_ERR_SHAPE;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    FitWs w = carve_fit(workspace, N, D, K);
+    const size_t KD = (size_t)K * D;
+    double *meanQ = w.meanQ, *meanF = w.meanF;
+    int32_t *labels = labels_out ? labels_out : w.a.labels;
+    float *C = centroids_out;
+
+    CAT_CUDA(launch_reset_control(w.a.ctl, s));
+    CAT_CUDA(cudaMemcpyAsync(C, init_centroids ? init_centroids : Yq, KD * sizeof(float),
+                             cudaMemcpyDeviceToDevice, s));
+
+    for (int t = 0; t < iters; ++t) {
+        st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s);
+        if (st != CAT_OK) return st;
+        st = run_cluster_sums(Yq, labels, N, D, K, w, w.sumQ, w.counts, s);
+        if (st != CAT_OK) return st;
+        CAT_CUDA(launch_centroids_from_sums(w.sumQ, w.counts, D, K, C, s));
+    }
+
+    // final assignment, then the closed form
+    st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s);
+    if (st != CAT_OK) return st;
+    st = run_cluster_sums(Yq, labels, N, D, K, w, w.sumQ, w.counts, s);
+    if (st != CAT_OK) return st;
+    st = run_cluster_sums(Yfp, labels, N, D, K, w, w.sumF, w.counts, s);
+    if (st != CAT_OK) return st;
+    CAT_CUDA(launch_means_from_sums(w.sumQ, w.counts, D, K, meanQ, s));
+    CAT_CUDA(launch_means_from_sums(w.sumF, w.counts, D, K, meanF, s));
+    st = run_centred(Yq, Yfp, labels, N, D, K, w, meanQ, meanF, w.var, w.cov, s);
+    if (st != CAT_OK) return st;
+    CAT_CUDA(launch_solve(w.sumQ, w.sumF, w.var, w.cov, w.counts, D, K, gamma_out, beta_out, s));
+    if (diag) CAT_CUDA(launch_fit_diag(w.a.ctl, w.counts, K, diag, s));
+    return CAT_OK;
+}
+
+cat_status_t cat_fit(const float *Yq, const float *Yfp, int64_t N, int32_t D, int32_t K,
+                     int32_t iters, float *centroids_out, float *gamma_out, float *beta_out,
+                     int32_t *labels_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return cat_fit_from(Yq, Yfp, N, D, K, iters, nullptr, centroids_out, gamma_out, beta_out,
+                        labels_out, nullptr, workspace, workspace_bytes, stream);
+}
+
+cat_status_t cat_cluster_sums(const float *Y, const int32_t *labels, int64_t N, int32_t D,
+                              int32_t K, double *sums_out, int64_t *counts_out, void *workspace,
+                              size_t workspace_bytes, void *stream)
+{
+    if (!Y || !labels || !sums_out || !counts_out) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (!aligned16(Y) || !aligned16(labels) || !aligned16(sums_out) || !aligned16(counts_out))
+        return CAT_ERR_ALIGN;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    FitWs w = carve_fit(workspace, N, D, K);
+    return run_cluster_sums(Y, labels, N, D, K, w, sums_out, counts_out,
+                            reinterpret_cast<cudaStream_t>(stream));
+}
+
+cat_status_t cat_centroids_from_sums(const double *sums, const int64_t *counts, int32_t D,
+                                     int32_t K, float *centroids_inout, void *stream)
+{
+    if (!sums || !counts || !centroids_inout) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(K, D, K, false);
+    if (st != CAT_OK) return st;
+    CAT_CUDA(launch_centroids_from_sums(sums, counts, D, K, centroids_inout,
+                                        reinterpret_cast<cudaStream_t>(stream)));
+    return CAT_OK;
+}
+
+cat_status_t cat_centred_moments(const float *Yq, const float *Yfp, const int32_t *labels,
+                                 int64_t N, int32_t D, int32_t K, const double *meanQ,
+                                 const double *meanF, double *var_out, double *cov_out,
+                                 void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!Yq || !Yfp || !labels || !meanQ || !meanF || !var_out || !cov_out) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (!aligned16(Yq) || !aligned16(Yfp) || !aligned16(labels) || !aligned16(meanQ) ||
+        !aligned16(meanF) || !aligned16(var_out) || !aligned16(cov_out))
+        return CAT_ERR_ALIGN;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    FitWs w = carve_fit(workspace, N, D, K);
+    return run_centred(Yq, Yfp, labels, N, D, K, w, meanQ, meanF, var_out, cov_out,
+                       reinterpret_cast<cudaStream_t>(stream));
+}
+
+cat_status_t cat_solve_gamma_beta(const double *sumQ, const double *sumF, const double *var_sum,
+                                  const double *cov_sum, const int64_t *counts, int32_t D,
+                                  int32_t K, float *gamma_out, float *beta_out, void *stream)
+{
+    if (!sumQ || !sumF || !var_sum || !cov_sum || !counts || !gamma_out || !beta_out)
+        return CAT_ERR_NULL;
+    cat_status_t st = check_shape(K, D, K, false);
+    if (st != CAT_OK) return st;
+    CAT_CUDA(launch_solve(sumQ, sumF, var_sum, cov_sum, counts, D, K, gamma_out, beta_out,
+                          reinterpret_cast<cudaStream_t>(stream)));
+    return CAT_OK;
+}
+
+const char *cat_status_string(cat_status_t status)
+{
+    switch (status) {
+    case CAT_OK: return "ok";
+    case CAT_ERR_NULL: return "a required pointer is NULL";
+    case CAT_ERR_SHAPE: return "bad shape or parameter (need N >= K >= 1, D >= 1, iters >= 0, 0 <= alpha <= 1)";
+    case CAT_ERR_ALIGN: return "a base pointer is not 16-byte aligned";
+    case CAT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case CAT_ERR_CUDA: return "a CUDA runtime call failed (see cat_last_cuda_error)";
+    case CAT_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+    case CAT_ERR_UNSUPPORTED: return "size beyond the supported limits (CAT_MAX_K, CAT_MAX_D, N < 2^31)";
+    default: return "unknown status";
+    }
+}
+
+int cat_last_cuda_error(void) { return g_last_cuda_error; }
+const char *cat_version(void) { return "cat-b200 0.1 (sm_100a)"; }
+int64_t cat_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,114 @@
+// Internal declarations shared by the translation units of libcat.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "cat.h"
+
+namespace cat {
+
+// ---------------------------------------------------------------- launch bookkeeping
+extern thread_local int g_last_cuda_error;
+void count_launch(int n = 1);
+
+inline bool cuda_ok(cudaError_t e)
+{
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return false;
+    }
+    return true;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---------------------------------------------------------------- workspace layouts
+// Control block at the start of every workspace (device memory).
+struct Control {
+    int32_t refine_count;        // rows queued for the exact fp64 pass by the current assignment
+    int32_t device_status;       // CAT_OK or CAT_ERR_DEVICE_TIMEOUT
+    int64_t refined_total;       // running total over assignments
+    int64_t refined_last;        // refine_count of the latest finished assignment
+    int64_t pad[5];
+};
+
+// Geometry of the segmented-sum kernels for one (N, D, K): identical in the
+// workspace query and at launch time.
+struct SumGeom {
+    int cpl;        // columns per lane: 1, 2 or 4 (slice width = 32*cpl)
+    int nacc;       // accumulator planes held in shared memory at once (1 or 2)
+    int copies;     // accumulator copies per cluster (spreads small K over the warps)
+    int nslices;    // column slices
+    int nchunks;    // row chunks
+    int64_t rows_per_chunk;
+    size_t smem_bytes;
+};
+SumGeom sum_geometry(int64_t N, int D, int K, int planes);
+
+struct AssignWs {          // what assign/apply need
+    Control *ctl;
+    float *cnorm;          // [K] squared centroid norms, fp32
+    int32_t *refine_rows;  // [N]
+    int32_t *labels;       // [N] (used when the caller passes no labels_out)
+    float *gamma_b;        // [K*D] blended gamma (alpha != 1)
+    float *beta_b;         // [K*D]
+    size_t bytes;
+};
+AssignWs carve_assign(void *base, int64_t N, int D, int K);
+
+struct FitWs {
+    AssignWs a;
+    double *partial;       // [nchunks][2][K*D] partial sums of the segmented kernels
+    int32_t *partial_cnt;  // [nchunks][K]
+    double *sumQ, *sumF, *var, *cov;   // [K*D] each
+    double *meanQ, *meanF;             // [K*D] each
+    int64_t *counts;       // [K]
+    size_t bytes;
+};
+FitWs carve_fit(void *base, int64_t N, int D, int K);
+
+// ---------------------------------------------------------------- kernel launchers (cat_kernels.cu)
+// All return a cudaError_t from the launch; none synchronises.
+
+// cnorm[k] = ||c_k||^2 (fp64 accumulate, rounded to fp32); also resets ctl->refine_count.
+cudaError_t launch_centroid_norms(const float *C, int D, int K, float *cnorm, Control *ctl,
+                                  cudaStream_t s);
+
+// Fast fp32 scores + certainty test; optional fused affine epilogue.
+cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *C,
+                          const float *cnorm, int32_t *labels, int32_t *refine_rows, Control *ctl,
+                          const float *gamma, const float *beta, float *out, cudaStream_t s);
+
+// Exact fp64 direct-form labels for the queued rows; optional affine output.
+cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *C,
+                          int32_t *labels, const int32_t *refine_rows, Control *ctl,
+                          const float *gamma, const float *beta, float *out, cudaStream_t s);
+
+// Segmented sums.  mode 0: partial[chunk][0] += Y rows per label (+ counts).
+// mode 1: centred moments: planes selected by mask (1 = var, 2 = cov).
+cudaError_t launch_cluster_partial(const float *Y, const float *F, const int32_t *labels,
+                                   int64_t N, int D, int K, const SumGeom &g,
+                                   const double *meanQ, const double *meanF, int mask,
+                                   double *partial, int32_t *partial_cnt, cudaStream_t s);
+
+// out[k*D+j] = sum over chunks of partial[chunk][plane][k*D+j]; counts likewise (may be NULL).
+cudaError_t launch_reduce_partials(const double *partial, const int32_t *partial_cnt, int nchunks,
+                                   int nplanes, int plane, int D, int K, double *out,
+                                   int64_t *counts, cudaStream_t s);
+
+cudaError_t launch_centroids_from_sums(const double *sums, const int64_t *counts, int D, int K,
+                                       float *C, cudaStream_t s);
+cudaError_t launch_means_from_sums(const double *sums, const int64_t *counts, int D, int K,
+                                   double *mean, cudaStream_t s);
+cudaError_t launch_solve(const double *sumQ, const double *sumF, const double *var,
+                         const double *cov, const int64_t *counts, int D, int K, float *gamma,
+                         float *beta, cudaStream_t s);
+cudaError_t launch_blend_params(const float *gamma, const float *beta, float alpha, int64_t KD,
+                                float *gamma_b, float *beta_b, cudaStream_t s);
+cudaError_t launch_fit_diag(const Control *ctl, const int64_t *counts, int K, cat_fit_diag_t *diag,
+                            cudaStream_t s);
+cudaError_t launch_reset_control(Control *ctl, cudaStream_t s);
+
+}  // namespace cat

@@ -1,0 +1,892 @@
+// CUDA kernels of the CAT hot path (sm_100a), general fp32 path.
+//
+//   centroid_norms_kernel   ||c_k||^2 for the expanded-form scores
+//   assign_kernel           nearest-centroid scores on the fp32 pipes + certainty test
+//                           (+ fused per-cluster affine epilogue for inference)
+//   refine_kernel           exact fp64 direct-form decision for the rows the fast
+//                           scores cannot separate
+//   cluster_partial_kernel  segmented (per-cluster) column sums / centred moments with
+//                           block-private fp64 accumulators in shared memory
+//   small element-wise kernels for centroid update, means and the gamma/beta solve
+//
+// Label decision rule.  The K-Means assignment step needs argmin_k ||y - c_k||^2
+// (lowest k on ties).  The fast pass evaluates t_k = ||c_k||^2 - 2 y.c_k in fp32,
+// whose error is bounded by
+//     e <= u * ((2D + 4) * ||y|| * cmax + 4 * cmax^2),  u = 2^-24, cmax = max_k ||c_k||
+// (D-term FMA chain, rounding of the stored norm, the final FMA).  If the two smallest
+// scores are further apart than 2e the fast argmin is the exact argmin.  Otherwise the
+// row is queued and decided by direct-form fp64 distances, scanning k upwards with a
+// strict '<' -- the same arithmetic a straightforward double-precision K-Means uses.
+#include "cat_internal.cuh"
+
+#include <math_constants.h>
+
+namespace cat {
+
+constexpr int kMaxDevices = 64;
+
+// ======================================================================================
+// small helpers
+// ======================================================================================
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src, int src_bytes)
+{
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem_src),
+                 "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ======================================================================================
+// centroid norms
+// ======================================================================================
+
+__global__ void centroid_norms_kernel(const float *__restrict__ C, int D, int K,
+                                      float *__restrict__ cnorm, Control *ctl)
+{
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (blockIdx.x == 0 && threadIdx.x == 0) ctl->refine_count = 0;
+    if (warp >= K) return;
+    const float *c = C + (size_t)warp * D;
+    double s = 0.0;
+    for (int j = lane; j < D; j += 32) {
+        double v = (double)c[j];
+        s += v * v;
+    }
+    s = warp_sum(s);
+    // round up so that the stored norm never under-states the true one
+    if (lane == 0) cnorm[warp] = __double2float_ru(s);
+}
+
+cudaError_t launch_centroid_norms(const float *C, int D, int K, float *cnorm, Control *ctl,
+                                  cudaStream_t s)
+{
+    int threads = 128;
+    int blocks = (K * 32 + threads - 1) / threads;
+    centroid_norms_kernel<<<blocks, threads, 0, s>>>(C, D, K, cnorm, ctl);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ======================================================================================
+// assignment (fast fp32 scores)
+// ======================================================================================
+
+constexpr int A_BM = 128;       // rows per CTA
+constexpr int A_BK = 16;        // D-slab per pipeline stage
+constexpr int A_LD = A_BK + 4;  // padded row stride in floats (5 x 16 B: conflict-free 128-bit reads)
+constexpr int A_STAGES = 3;
+constexpr int A_THREADS = 128;
+
+struct AssignParams {
+    const float *Y;
+    const float *C;
+    const float *cnorm;
+    int32_t *labels;
+    int32_t *refine_rows;
+    Control *ctl;
+    const float *gamma;
+    const float *beta;
+    float *out;
+    int64_t N;
+    int D;
+    int K;
+};
+
+template <int BN>
+struct AssignSmem {
+    float a[A_STAGES][A_BM * A_LD];
+    float b[A_STAGES][BN * A_LD];
+    float red[4];
+    float best[A_BM];
+    float second[A_BM];
+    int idx[A_BM];
+    int lab[A_BM];
+};
+
+template <int BN, bool VEC4>
+__device__ __forceinline__ void assign_load_tile(AssignSmem<BN> &sm, int stage, const AssignParams &p,
+                                                 int64_t row0, int chunk, int k0, int tid)
+{
+    float *As = sm.a[stage];
+    float *Bs = sm.b[stage];
+    if (VEC4) {
+#pragma unroll
+        for (int q = 0; q < (A_BM * A_BK / 4) / A_THREADS; ++q) {
+            int e = tid + q * A_THREADS;
+            int r = e >> 2, c4 = e & 3;
+            int col = k0 + c4 * 4;
+            int64_t row = row0 + r;
+            bool ok = (row < p.N) && (col < p.D);
+            const float *src = ok ? (p.Y + (size_t)row * p.D + col) : p.Y;
+            cp_async16(As + r * A_LD + c4 * 4, src, ok ? 16 : 0);
+        }
+        for (int e = tid; e < BN * A_BK / 4; e += A_THREADS) {
+            int n = e >> 2, c4 = e & 3;
+            int col = k0 + c4 * 4;
+            int k = chunk * BN + n;
+            bool ok = (k < p.K) && (col < p.D);
+            const float *src = ok ? (p.C + (size_t)k * p.D + col) : p.C;
+            cp_async16(Bs + n * A_LD + c4 * 4, src, ok ? 16 : 0);
+        }
+    } else {
+        for (int e = tid; e < A_BM * A_BK; e += A_THREADS) {
+            int r = e / A_BK, c = e % A_BK;
+            int col = k0 + c;
+            int64_t row = row0 + r;
+            As[r * A_LD + c] = (row < p.N && col < p.D) ? p.Y[(size_t)row * p.D + col] : 0.f;
+        }
+        for (int e = tid; e < BN * A_BK; e += A_THREADS) {
+            int n = e / A_BK, c = e % A_BK;
+            int col = k0 + c;
+            int k = chunk * BN + n;
+            Bs[n * A_LD + c] = (k < p.K && col < p.D) ? p.C[(size_t)k * p.D + col] : 0.f;
+        }
+    }
+}
+
+// BN centroids per chunk, 8 per thread; TX = BN/8 threads share a row; each thread owns
+// TM = TX rows (row = ty + TY*i) so that a CTA always covers 128 rows.
+template <int BN, bool VEC4, bool AFFINE>
+__global__ void __launch_bounds__(A_THREADS) assign_kernel(AssignParams p)
+{
+    constexpr int TX = BN / 8;
+    constexpr int TY = A_THREADS / TX;
+    constexpr int TM = A_BM / TY;
+    static_assert(TM == TX, "tile shape");
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    AssignSmem<BN> &sm = *reinterpret_cast<AssignSmem<BN> *>(smem_raw);
+
+    const int tid = threadIdx.x;
+    const int tx = tid % TX;
+    const int ty = tid / TX;
+    const int64_t row0 = (int64_t)blockIdx.x * A_BM;
+
+    // cmax^2 = max_k ||c_k||^2
+    {
+        float m = 0.f;
+        for (int k = tid; k < p.K; k += A_THREADS) m = fmaxf(m, p.cnorm[k]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if ((tid & 31) == 0) sm.red[tid >> 5] = m;
+    }
+
+    const int ktiles = (p.D + A_BK - 1) / A_BK;
+    const int nchunks = (p.K + BN - 1) / BN;
+    const int T = ktiles * nchunks;
+
+    for (int s = 0; s < A_STAGES - 1; ++s) {
+        if (s < T) assign_load_tile<BN, VEC4>(sm, s, p, row0, s / ktiles, (s % ktiles) * A_BK, tid);
+        cp_async_commit();
+    }
+
+    float acc[TM][8];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+
+    float rb1[TM], rb2[TM];
+    int ridx[TM];
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+        rb1[i] = CUDART_INF_F;
+        rb2[i] = CUDART_INF_F;
+        ridx[i] = 0;
+    }
+    float ysq = 0.f;  // ||y_row||^2 of row `tid`, accumulated during the first chunk
+
+    int chunk = 0, kt = 0;
+    for (int t = 0; t < T; ++t) {
+        cp_async_wait<A_STAGES - 2>();
+        __syncthreads();
+        {
+            int tn = t + A_STAGES - 1;
+            if (tn < T)
+                assign_load_tile<BN, VEC4>(sm, tn % A_STAGES, p, row0, tn / ktiles,
+                                           (tn % ktiles) * A_BK, tid);
+            cp_async_commit();
+        }
+        const float *As = sm.a[t % A_STAGES];
+        const float *Bs = sm.b[t % A_STAGES];
+
+        if (chunk == 0) {
+#pragma unroll
+            for (int kk = 0; kk < A_BK; kk += 4) {
+                float4 v = *reinterpret_cast<const float4 *>(As + tid * A_LD + kk);
+                ysq = fmaf(v.x, v.x, ysq);
+                ysq = fmaf(v.y, v.y, ysq);
+                ysq = fmaf(v.z, v.z, ysq);
+                ysq = fmaf(v.w, v.w, ysq);
+            }
+        }
+
+#pragma unroll
+        for (int kk = 0; kk < A_BK; kk += 4) {
+            float4 a[TM];
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+                a[i] = *reinterpret_cast<const float4 *>(As + (ty + TY * i) * A_LD + kk);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float4 b = *reinterpret_cast<const float4 *>(Bs + (tx + TX * j) * A_LD + kk);
+#pragma unroll
+                for (int i = 0; i < TM; ++i) {
+                    acc[i][j] = fmaf(a[i].x, b.x, acc[i][j]);
+                    acc[i][j] = fmaf(a[i].y, b.y, acc[i][j]);
+                    acc[i][j] = fmaf(a[i].z, b.z, acc[i][j]);
+                    acc[i][j] = fmaf(a[i].w, b.w, acc[i][j]);
+                }
+            }
+        }
+
+        if (++kt == ktiles) {
+            // scores of this chunk of centroids: t = ||c||^2 - 2 y.c
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                int n = chunk * BN + tx + TX * j;
+                float cn = (n < p.K) ? p.cnorm[n] : CUDART_INF_F;
+#pragma unroll
+                for (int i = 0; i < TM; ++i) {
+                    float sc = (n < p.K) ? fmaf(-2.f, acc[i][j], cn) : CUDART_INF_F;
+                    if (sc < rb1[i]) {
+                        rb2[i] = rb1[i];
+                        rb1[i] = sc;
+                        ridx[i] = n;
+                    } else if (sc < rb2[i]) {
+                        rb2[i] = sc;
+                    }
+                    acc[i][j] = 0.f;
+                }
+            }
+            kt = 0;
+            ++chunk;
+        }
+    }
+    cp_async_wait<0>();
+
+    // merge the TX threads that share a row
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+#pragma unroll
+        for (int o = 1; o < TX; o <<= 1) {
+            float ob1 = __shfl_xor_sync(0xffffffffu, rb1[i], o);
+            float ob2 = __shfl_xor_sync(0xffffffffu, rb2[i], o);
+            int oidx = __shfl_xor_sync(0xffffffffu, ridx[i], o);
+            bool take = (ob1 < rb1[i]) || (ob1 == rb1[i] && oidx < ridx[i]);
+            float hi = take ? rb1[i] : ob1;  // the larger of the two bests
+            rb2[i] = fminf(fminf(rb2[i], ob2), hi);
+            if (take) {
+                rb1[i] = ob1;
+                ridx[i] = oidx;
+            }
+        }
+        if (tx == 0) {
+            int r = ty + TY * i;
+            sm.best[r] = rb1[i];
+            sm.second[r] = rb2[i];
+            sm.idx[r] = ridx[i];
+        }
+    }
+    __syncthreads();
+
+    {
+        const float cmax2 = fmaxf(fmaxf(sm.red[0], sm.red[1]), fmaxf(sm.red[2], sm.red[3]));
+        const int64_t row = row0 + tid;
+        int lab = -1;
+        if (row < p.N) {
+            const float u = 5.9604645e-8f;  // 2^-24
+            float e = 1.0625f * u *
+                      ((2.f * (float)p.D + 4.f) * sqrtf(ysq) * sqrtf(cmax2) + 4.f * cmax2);
+            float gap = sm.second[tid] - sm.best[tid];
+            int k = sm.idx[tid];
+            bool certain = (p.K == 1) || (gap > 2.f * e);
+            p.labels[row] = k;
+            if (certain) {
+                lab = k;
+            } else {
+                int slot = atomicAdd(&p.ctl->refine_count, 1);
+                p.refine_rows[slot] = (int32_t)row;
+            }
+        }
+        sm.lab[tid] = lab;
+    }
+
+    if (AFFINE) {
+        __syncthreads();
+        if (VEC4) {
+            const int D4 = p.D >> 2;
+            const float4 *Y4 = reinterpret_cast<const float4 *>(p.Y);
+            const float4 *G4 = reinterpret_cast<const float4 *>(p.gamma);
+            const float4 *B4 = reinterpret_cast<const float4 *>(p.beta);
+            float4 *O4 = reinterpret_cast<float4 *>(p.out);
+            for (int r = 0; r < A_BM; r += 4) {
+                for (int c = tid; c < D4; c += A_THREADS) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        int l = sm.lab[r + q];
+                        if (l < 0) continue;
+                        size_t o = (size_t)(row0 + r + q) * D4 + c;
+                        float4 y = __ldcs(Y4 + o);
+                        float4 g = __ldg(G4 + (size_t)l * D4 + c);
+                        float4 b = __ldg(B4 + (size_t)l * D4 + c);
+                        float4 v;
+                        v.x = fmaf(g.x, y.x, b.x);
+                        v.y = fmaf(g.y, y.y, b.y);
+                        v.z = fmaf(g.z, y.z, b.z);
+                        v.w = fmaf(g.w, y.w, b.w);
+                        __stcs(O4 + o, v);
+                    }
+                }
+            }
+        } else {
+            for (int r = 0; r < A_BM; ++r) {
+                int l = sm.lab[r];
+                if (l < 0) continue;
+                size_t o = (size_t)(row0 + r) * p.D;
+                for (int c = tid; c < p.D; c += A_THREADS)
+                    p.out[o + c] = fmaf(p.gamma[(size_t)l * p.D + c], p.Y[o + c],
+                                        p.beta[(size_t)l * p.D + c]);
+            }
+        }
+    }
+}
+
+template <int BN, bool VEC4, bool AFFINE>
+static cudaError_t launch_assign_t(const AssignParams &p, cudaStream_t s)
+{
+    auto kern = assign_kernel<BN, VEC4, AFFINE>;
+    size_t smem = sizeof(AssignSmem<BN>);
+    static bool configured[kMaxDevices] = {};  // the attribute is kept per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = -1;
+    if (dev < 0 || !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0) configured[dev] = true;
+    }
+    unsigned blocks = (unsigned)((p.N + A_BM - 1) / A_BM);
+    kern<<<blocks, A_THREADS, smem, s>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <bool VEC4, bool AFFINE>
+static cudaError_t launch_assign_bn(const AssignParams &p, cudaStream_t s)
+{
+    if (p.K <= 8) return launch_assign_t<8, VEC4, AFFINE>(p, s);
+    if (p.K <= 16) return launch_assign_t<16, VEC4, AFFINE>(p, s);
+    if (p.K <= 32) return launch_assign_t<32, VEC4, AFFINE>(p, s);
+    return launch_assign_t<64, VEC4, AFFINE>(p, s);
+}
+
+cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *C,
+                          const float *cnorm, int32_t *labels, int32_t *refine_rows, Control *ctl,
+                          const float *gamma, const float *beta, float *out, cudaStream_t s)
+{
+    AssignParams p{Y, C, cnorm, labels, refine_rows, ctl, gamma, beta, out, N, D, K};
+    const bool vec = (D % 4 == 0);
+    const bool affine = (out != nullptr);
+    if (vec) return affine ? launch_assign_bn<true, true>(p, s) : launch_assign_bn<true, false>(p, s);
+    return affine ? launch_assign_bn<false, true>(p, s) : launch_assign_bn<false, false>(p, s);
+}
+
+// ======================================================================================
+// exact decision for queued rows
+// ======================================================================================
+
+constexpr int R_THREADS = 128;
+
+template <bool AFFINE>
+__global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restrict__ Y, int64_t N,
+                                                           int D, int K, const float *__restrict__ C,
+                                                           int32_t *labels,
+                                                           const int32_t *__restrict__ refine_rows,
+                                                           Control *ctl, const float *gamma,
+                                                           const float *beta, float *out)
+{
+    int count = ctl->refine_count;
+    if ((int64_t)count > N) count = (int)N;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctl->refined_total += count;
+        ctl->refined_last = count;
+    }
+    const int lane = threadIdx.x & 31;
+    const int warps_per_block = R_THREADS / 32;
+    const int gw = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+    const int nw = gridDim.x * warps_per_block;
+    for (int it = gw; it < count; it += nw) {
+        int64_t row = refine_rows[it];
+        if (row < 0 || row >= N) continue;
+        const float *y = Y + (size_t)row * D;
+        double best = CUDART_INF;
+        int bk = 0;
+        for (int k = 0; k < K; ++k) {
+            const float *c = C + (size_t)k * D;
+            double s = 0.0;
+            for (int j = lane; j < D; j += 32) {
+                double d = (double)y[j] - (double)c[j];
+                s = fma(d, d, s);
+            }
+            s = warp_sum(s);
+            if (s < best) {
+                best = s;
+                bk = k;
+            }
+        }
+        if (lane == 0) labels[row] = bk;
+        if (AFFINE) {
+            const float *g = gamma + (size_t)bk * D;
+            const float *b = beta + (size_t)bk * D;
+            float *o = out + (size_t)row * D;
+            for (int j = lane; j < D; j += 32) o[j] = fmaf(g[j], y[j], b[j]);
+        }
+    }
+}
+
+cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *C,
+                          int32_t *labels, const int32_t *refine_rows, Control *ctl,
+                          const float *gamma, const float *beta, float *out, cudaStream_t s)
+{
+    int64_t want = (N + (R_THREADS / 32) - 1) / (R_THREADS / 32);
+    int blocks = (int)(want < 592 ? want : 592);
+    if (out)
+        refine_kernel<true><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
+                                                         gamma, beta, out);
+    else
+        refine_kernel<false><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
+                                                          gamma, beta, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ======================================================================================
+// segmented sums with block-private accumulators
+// ======================================================================================
+
+constexpr int S_THREADS = 512;
+constexpr int S_WARPS = S_THREADS / 32;
+constexpr int S_LABELS = 2048;               // labels staged per batch
+constexpr size_t S_ACC_BUDGET = 160 * 1024;  // bytes of shared memory for accumulators
+
+SumGeom sum_geometry(int64_t N, int D, int K, int planes)
+{
+    SumGeom g{};
+    g.copies = (K >= 4 * S_WARPS) ? 1 : (4 * S_WARPS + K - 1) / K;
+    const size_t kg = (size_t)K * g.copies;
+    g.nacc = planes;
+    g.cpl = 0;
+    for (int pass = 0; pass < 2 && g.cpl == 0; ++pass) {
+        for (int cpl = 4; cpl >= 1; cpl >>= 1) {
+            if (D % cpl) continue;
+            if (kg * 32 * cpl * sizeof(double) * g.nacc <= S_ACC_BUDGET) {
+                g.cpl = cpl;
+                break;
+            }
+        }
+        if (g.cpl == 0) g.nacc = 1;  // one plane at a time
+    }
+    if (g.cpl == 0) g.cpl = 1;  // unreachable for K <= CAT_MAX_K
+    const int sw = 32 * g.cpl;
+    g.nslices = (D + sw - 1) / sw;
+    int64_t maxchunks = (N + 255) / 256;
+    int64_t want = (296 + g.nslices - 1) / g.nslices;
+    int64_t nch = want < 1 ? 1 : want;
+    if (nch > 32) nch = 32;
+    if (nch > maxchunks) nch = maxchunks;
+    if (nch < 1) nch = 1;
+    g.nchunks = (int)nch;
+    g.rows_per_chunk = (N + nch - 1) / nch;
+    g.smem_bytes = kg * sw * sizeof(double) * g.nacc + kg * sizeof(int) + S_LABELS * sizeof(int);
+    return g;
+}
+
+struct SumParams {
+    const float *Y;
+    const float *F;
+    const int32_t *labels;
+    const double *meanQ;
+    const double *meanF;
+    double *partial;
+    int32_t *partial_cnt;
+    int64_t N;
+    int64_t rows_per_chunk;
+    int D;
+    int K;
+    int copies;
+    int mask;
+};
+
+template <int CPL>
+__device__ __forceinline__ void load_cols(const float *src, float (&v)[CPL])
+{
+    if constexpr (CPL == 4) {
+        float4 t = __ldg(reinterpret_cast<const float4 *>(src));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else if constexpr (CPL == 2) {
+        float2 t = __ldg(reinterpret_cast<const float2 *>(src));
+        v[0] = t.x; v[1] = t.y;
+    } else {
+        v[0] = __ldg(src);
+    }
+}
+
+// One CTA = (column slice, row chunk).  Warp w owns the accumulator rows v with
+// v % S_WARPS == w, where v = label * copies + row % copies, so no two warps ever touch
+// the same accumulator and every sum is formed in ascending row order.
+template <int CPL, int NACC, bool CENTRED>
+__global__ void __launch_bounds__(S_THREADS) cluster_partial_kernel(SumParams p)
+{
+    constexpr int SW = 32 * CPL;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int KG = p.K * p.copies;
+    double *acc = reinterpret_cast<double *>(smem_raw);               // [NACC][KG][SW]
+    int *cnt = reinterpret_cast<int *>(acc + (size_t)NACC * KG * SW);  // [KG]
+    int *lab_s = cnt + KG;                                            // [S_LABELS]
+
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int slice = blockIdx.x, chunk = blockIdx.y;
+    const int col = slice * SW + lane * CPL;
+    const bool col_ok = col < p.D;
+
+    for (int e = tid; e < NACC * KG * SW; e += S_THREADS) acc[e] = 0.0;
+    for (int e = tid; e < KG; e += S_THREADS) cnt[e] = 0;
+
+    const int64_t r_begin = (int64_t)chunk * p.rows_per_chunk;
+    int64_t r_end = r_begin + p.rows_per_chunk;
+    if (r_end > p.N) r_end = p.N;
+
+    for (int64_t b = r_begin; b < r_end; b += S_LABELS) {
+        __syncthreads();
+        for (int e = tid; e < S_LABELS; e += S_THREADS) {
+            int64_t r = b + e;
+            int l = (r < r_end) ? p.labels[r] : -1;
+            lab_s[e] = (l >= 0 && l < p.K) ? l : -1;
+        }
+        __syncthreads();
+        int nb = (int)((r_end - b < S_LABELS) ? (r_end - b) : S_LABELS);
+        for (int base = 0; base < nb; base += 32) {
+            int l = lab_s[base + lane];
+            int64_t row = b + base + lane;
+            int v = (l >= 0) ? l * p.copies + (int)(row % p.copies) : -1;
+            unsigned m = __ballot_sync(0xffffffffu, v >= 0 && (v % S_WARPS) == w);
+            while (m) {
+                int vv[4];
+                int64_t rr[4];
+                float q[4][CPL], f[4][CPL];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (m) {
+                        int bit = __ffs(m) - 1;
+                        m &= m - 1;
+                        vv[u] = __shfl_sync(0xffffffffu, v, bit);
+                        rr[u] = b + base + bit;
+                    } else {
+                        vv[u] = -1;
+                        rr[u] = 0;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (vv[u] >= 0 && col_ok) {
+                        const float *src = p.Y + (size_t)rr[u] * p.D + col;
+                        load_cols<CPL>(src, q[u]);
+                        if (CENTRED) {
+                            const float *srf = p.F + (size_t)rr[u] * p.D + col;
+                            load_cols<CPL>(srf, f[u]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (vv[u] < 0) continue;
+                    if (!CENTRED && lane == 0 && slice == 0) cnt[vv[u]]++;
+                    if (!col_ok) continue;
+                    double *a0 = acc + ((size_t)vv[u] * SW + lane * CPL);
+                    if (!CENTRED) {
+#pragma unroll
+                        for (int c = 0; c < CPL; ++c) a0[c] += (double)q[u][c];
+                    } else {
+                        int l = vv[u] / p.copies;
+                        const double *mq = p.meanQ + (size_t)l * p.D + col;
+                        const double *mf = p.meanF + (size_t)l * p.D + col;
+#pragma unroll
+                        for (int c = 0; c < CPL; ++c) {
+                            double dq = (double)q[u][c] - mq[c];
+                            double df = (double)f[u][c] - mf[c];
+                            if (NACC == 2) {
+                                a0[c] = fma(dq, dq, a0[c]);
+                                a0[(size_t)KG * SW + c] = fma(dq, df, a0[(size_t)KG * SW + c]);
+                            } else if (p.mask == 1) {
+                                a0[c] = fma(dq, dq, a0[c]);
+                            } else {
+                                a0[c] = fma(dq, df, a0[c]);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    // fold the copies and publish this CTA's partial sums
+    const size_t KD = (size_t)p.K * p.D;
+    for (int e = tid; e < NACC * p.K * SW; e += S_THREADS) {
+        int a = e / (p.K * SW);
+        int rem = e - a * (p.K * SW);
+        int k = rem / SW, c = rem - k * SW;
+        int gc = slice * SW + c;
+        if (gc >= p.D) continue;
+        double s = 0.0;
+        for (int g = 0; g < p.copies; ++g) s += acc[((size_t)a * KG + (size_t)k * p.copies + g) * SW + c];
+        int plane = (NACC == 2) ? a : ((CENTRED && p.mask == 2) ? 1 : 0);
+        p.partial[((size_t)chunk * 2 + plane) * KD + (size_t)k * p.D + gc] = s;
+    }
+    if (!CENTRED && slice == 0) {
+        for (int k = tid; k < p.K; k += S_THREADS) {
+            int s = 0;
+            for (int g = 0; g < p.copies; ++g) s += cnt[k * p.copies + g];
+            p.partial_cnt[(size_t)chunk * p.K + k] = s;
+        }
+    }
+}
+
+template <int CPL, int NACC, bool CENTRED>
+static cudaError_t launch_partial_t(const SumParams &p, const SumGeom &g, cudaStream_t s)
+{
+    auto kern = cluster_partial_kernel<CPL, NACC, CENTRED>;
+    static size_t configured[kMaxDevices] = {};  // the attribute is kept per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = -1;
+    if (dev < 0 || g.smem_bytes > configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)g.smem_bytes);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0) configured[dev] = g.smem_bytes;
+    }
+    dim3 grid((unsigned)g.nslices, (unsigned)g.nchunks);
+    kern<<<grid, S_THREADS, g.smem_bytes, s>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cluster_partial(const float *Y, const float *F, const int32_t *labels,
+                                   int64_t N, int D, int K, const SumGeom &g,
+                                   const double *meanQ, const double *meanF, int mask,
+                                   double *partial, int32_t *partial_cnt, cudaStream_t s)
+{
+    SumParams p{Y, F, labels, meanQ, meanF, partial, partial_cnt, N, g.rows_per_chunk,
+                D, K, g.copies, mask};
+    const bool centred = (mask != 0);
+    if (!centred) {
+        switch (g.cpl) {
+        case 4: return launch_partial_t<4, 1, false>(p, g, s);
+        case 2: return launch_partial_t<2, 1, false>(p, g, s);
+        default: return launch_partial_t<1, 1, false>(p, g, s);
+        }
+    }
+    if (g.nacc == 2) {
+        switch (g.cpl) {
+        case 4: return launch_partial_t<4, 2, true>(p, g, s);
+        case 2: return launch_partial_t<2, 2, true>(p, g, s);
+        default: return launch_partial_t<1, 2, true>(p, g, s);
+        }
+    }
+    switch (g.cpl) {
+    case 4: return launch_partial_t<4, 1, true>(p, g, s);
+    case 2: return launch_partial_t<2, 1, true>(p, g, s);
+    default: return launch_partial_t<1, 1, true>(p, g, s);
+    }
+}
+
+// ======================================================================================
+// element-wise kernels
+// ======================================================================================
+
+__global__ void reduce_partials_kernel(const double *__restrict__ partial,
+                                       const int32_t *__restrict__ partial_cnt, int nchunks,
+                                       int plane, size_t KD, int K, double *__restrict__ out,
+                                       int64_t *__restrict__ counts)
+{
+    size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < KD) {
+        double s = 0.0;
+        for (int c = 0; c < nchunks; ++c) s += partial[((size_t)c * 2 + plane) * KD + e];
+        out[e] = s;
+    }
+    if (counts && e < (size_t)K) {
+        int64_t s = 0;
+        for (int c = 0; c < nchunks; ++c) s += partial_cnt[(size_t)c * K + e];
+        counts[e] = s;
+    }
+}
+
+cudaError_t launch_reduce_partials(const double *partial, const int32_t *partial_cnt, int nchunks,
+                                   int nplanes, int plane, int D, int K, double *out,
+                                   int64_t *counts, cudaStream_t s)
+{
+    (void)nplanes;
+    size_t KD = (size_t)K * D;
+    int threads = 256;
+    unsigned blocks = (unsigned)((KD + threads - 1) / threads);
+    reduce_partials_kernel<<<blocks, threads, 0, s>>>(partial, partial_cnt, nchunks, plane, KD, K,
+                                                      out, counts);
+    count_launch();
+    return cudaGetLastError();
+}
+
+__global__ void centroids_from_sums_kernel(const double *__restrict__ sums,
+                                           const int64_t *__restrict__ counts, int D, size_t KD,
+                                           float *__restrict__ C)
+{
+    size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= KD) return;
+    int64_t n = counts[e / D];
+    if (n > 0) C[e] = (float)(sums[e] / (double)n);
+}
+
+cudaError_t launch_centroids_from_sums(const double *sums, const int64_t *counts, int D, int K,
+                                       float *C, cudaStream_t s)
+{
+    size_t KD = (size_t)K * D;
+    int threads = 256;
+    unsigned blocks = (unsigned)((KD + threads - 1) / threads);
+    centroids_from_sums_kernel<<<blocks, threads, 0, s>>>(sums, counts, D, KD, C);
+    count_launch();
+    return cudaGetLastError();
+}
+
+__global__ void means_from_sums_kernel(const double *__restrict__ sums,
+                                       const int64_t *__restrict__ counts, int D, size_t KD,
+                                       double *__restrict__ mean)
+{
+    size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= KD) return;
+    int64_t n = counts[e / D];
+    mean[e] = (n > 0) ? sums[e] / (double)n : 0.0;
+}
+
+cudaError_t launch_means_from_sums(const double *sums, const int64_t *counts, int D, int K,
+                                   double *mean, cudaStream_t s)
+{
+    size_t KD = (size_t)K * D;
+    int threads = 256;
+    unsigned blocks = (unsigned)((KD + threads - 1) / threads);
+    means_from_sums_kernel<<<blocks, threads, 0, s>>>(sums, counts, D, KD, mean);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// gamma = (cov/n) / max(var/n, 1e-8), beta = muF - gamma*muQ; empty cluster -> (1, 0).
+__global__ void solve_kernel(const double *__restrict__ sumQ, const double *__restrict__ sumF,
+                             const double *__restrict__ var, const double *__restrict__ cov,
+                             const int64_t *__restrict__ counts, int D, size_t KD,
+                             float *__restrict__ gamma, float *__restrict__ beta)
+{
+    size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= KD) return;
+    int64_t n = counts[e / D];
+    if (n <= 0) {
+        gamma[e] = 1.f;
+        beta[e] = 0.f;
+        return;
+    }
+    double dn = (double)n;
+    double v = var[e] / dn;
+    double c = cov[e] / dn;
+    if (v < 1e-8) v = 1e-8;
+    double g = c / v;
+    double b = sumF[e] / dn - g * (sumQ[e] / dn);
+    gamma[e] = (float)g;
+    beta[e] = (float)b;
+}
+
+cudaError_t launch_solve(const double *sumQ, const double *sumF, const double *var,
+                         const double *cov, const int64_t *counts, int D, int K, float *gamma,
+                         float *beta, cudaStream_t s)
+{
+    size_t KD = (size_t)K * D;
+    int threads = 256;
+    unsigned blocks = (unsigned)((KD + threads - 1) / threads);
+    solve_kernel<<<blocks, threads, 0, s>>>(sumQ, sumF, var, cov, counts, D, KD, gamma, beta);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// gamma' = 1 + alpha (gamma - 1), beta' = alpha beta  (so that gamma' y + beta' is the blend)
+__global__ void blend_params_kernel(const float *__restrict__ gamma, const float *__restrict__ beta,
+                                    double alpha, size_t KD, float *__restrict__ gb,
+                                    float *__restrict__ bb)
+{
+    size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= KD) return;
+    gb[e] = (float)(1.0 + alpha * ((double)gamma[e] - 1.0));
+    bb[e] = (float)(alpha * (double)beta[e]);
+}
+
+cudaError_t launch_blend_params(const float *gamma, const float *beta, float alpha, int64_t KD,
+                                float *gamma_b, float *beta_b, cudaStream_t s)
+{
+    int threads = 256;
+    unsigned blocks = (unsigned)((KD + threads - 1) / threads);
+    blend_params_kernel<<<blocks, threads, 0, s>>>(gamma, beta, (double)alpha, (size_t)KD, gamma_b,
+                                                   beta_b);
+    count_launch();
+    return cudaGetLastError();
+}
+
+__global__ void fit_diag_kernel(const Control *ctl, const int64_t *counts, int K,
+                                cat_fit_diag_t *diag)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int64_t empty = 0;
+    for (int k = 0; k < K; ++k) empty += (counts[k] == 0);
+    diag->refined_rows_total = ctl->refined_total;
+    diag->refined_rows_final = ctl->refined_last;
+    diag->empty_clusters_final = empty;
+    diag->device_status = ctl->device_status;
+}
+
+cudaError_t launch_fit_diag(const Control *ctl, const int64_t *counts, int K, cat_fit_diag_t *diag,
+                            cudaStream_t s)
+{
+    fit_diag_kernel<<<1, 32, 0, s>>>(ctl, counts, K, diag);
+    count_launch();
+    return cudaGetLastError();
+}
+
+__global__ void reset_control_kernel(Control *ctl)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        ctl->refine_count = 0;
+        ctl->device_status = CAT_OK;
+        ctl->refined_total = 0;
+        ctl->refined_last = 0;
+    }
+}
+
+cudaError_t launch_reset_control(Control *ctl, cudaStream_t s)
+{
+    reset_control_kernel<<<1, 32, 0, s>>>(ctl);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace cat

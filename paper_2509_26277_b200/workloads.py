@@ -175,19 +175,22 @@ def gaussian_mixture(name: str, config: int, seed: int, n: int, d: int, componen
     return Workload(name, config, K, iters, Yq[:n_fit], Yfp_fit, Yq)
 
 
-def make(config: int, device="cpu", rows_scale: float = 1.0) -> Workload:
+def make(config: int, device="cpu", rows_scale: float = 1.0, seed_offset: int = 0) -> Workload:
     """Build workload `config` (0-4) on `device`.
 
     rows_scale < 1 shrinks the row counts (never below K) for CPU-sized test
-    cases; shapes D, K, iters and the value recipe stay as specified."""
+    cases; shapes D, K, iters and the value recipe stay as specified.
+    seed_offset draws different rows from the same recipe (one shard per rank)."""
     if config in _LINEAR:
         name, seed, din, d, wb, ab, n_fit, n_apply, K, iters = _LINEAR[config]
+        seed += seed_offset
         n_fit = max(K, int(round(n_fit * rows_scale)))
         if n_apply is not None:
             n_apply = max(1, int(round(n_apply * rows_scale)))
         return linear_head(name, config, seed, din, d, wb, ab, n_fit, n_apply, K, iters, device)
     if config == 4:
         name, seed, n, d, comps, n_fit, K, iters = _MIXTURE
+        seed += seed_offset
         n = max(K, int(round(n * rows_scale)))
         n_fit = max(K, min(n, int(round(n_fit * rows_scale))))
         return gaussian_mixture(name, config, seed, n, d, comps, n_fit, K, iters, device)

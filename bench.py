@@ -246,6 +246,8 @@ def run_cuda(args):
     barrier()
     t_wall = time.perf_counter() - t_wall0
     launches = B.cat_kernel_launches() - launches0
+    rep_fit = B.cat_workspace_report(ws_fit) if world == 1 else None
+    rep_apply = B.cat_workspace_report(ws_apply)
     clocks = sampler.stop() if rank == 0 else None
 
     fit_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]
@@ -302,6 +304,8 @@ def run_cuda(args):
                          "peak_source": peak_src, "traffic": None},
             "roofline_fit": {"bound": "hbm", "kernel": "one Lloyd round of cat_fit (assign + segmented sums)",
                              "achieved": lloyd_gbs, "peak": peak, "unit": "GB/s", "frac": lloyd_gbs / peak},
+            "exact_pass_rows": {"apply": rep_apply["refined_rows_last"],
+                                "fit_all_assignments": rep_fit["refined_rows_total"] if rep_fit else None},
             "cpu_baseline": cpu_baseline,
             "e2e": e2e,
             "gpu_launches": int(launches),

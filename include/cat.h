@@ -192,6 +192,14 @@ cat_status_t cat_fit_host(const float *Yq_host, const float *Yfp_host, int64_t N
 
 /* ---- misc --------------------------------------------------------------- */
 
+/* Reads back counters kept in a workspace by the calls that used it last: waits for
+ * `stream`, then copies to the HOST pointers (each may be NULL) the number of rows
+ * whose label needed the exact fp64 pass in the latest assignment, the running
+ * total since the last cat_fit started on that workspace, and the device status
+ * word (CAT_OK or CAT_ERR_DEVICE_TIMEOUT). */
+cat_status_t cat_workspace_report(const void *workspace, void *stream, int64_t *refined_last_host,
+                                  int64_t *refined_total_host, int32_t *device_status_host);
+
 const char *cat_status_string(cat_status_t status);
 int cat_last_cuda_error(void);           /* cudaError_t of the last failing runtime call on this thread */
 const char *cat_version(void);

@@ -28,7 +28,8 @@ EXPORTS = [
     "cat_fit_workspace_bytes", "cat_fit", "cat_fit_from", "cat_apply_workspace_bytes",
     "cat_apply", "cat_apply_blend", "cat_assign", "cat_cluster_sums", "cat_centroids_from_sums",
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
-    "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_status_string",
+    "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
+    "cat_status_string",
     "cat_last_cuda_error", "cat_version", "cat_kernel_launches",
 ]
 
@@ -87,6 +88,8 @@ def lib():
                  "cat_cluster_sums", "cat_centroids_from_sums", "cat_centred_moments",
                  "cat_solve_gamma_beta", "cat_apply_host", "cat_fit_host"):
         getattr(L, name).restype = ctypes.c_int
+    L.cat_workspace_report.argtypes = [vp, vp, vp, vp, vp]
+    L.cat_workspace_report.restype = ctypes.c_int
     L.cat_status_string.argtypes = [ctypes.c_int]
     L.cat_status_string.restype = ctypes.c_char_p
     L.cat_last_cuda_error.restype = ctypes.c_int
@@ -319,6 +322,15 @@ def cat_fit_host(Yq_host, Yfp_host, K: int, iters: int, C_host, G_host, B_host, 
                             ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream())
     _check(st, "cat_fit_host")
     return C_host, G_host, B_host
+
+
+def cat_workspace_report(ws) -> dict:
+    """Counters of the calls that last used workspace `ws` (synchronises the current stream)."""
+    last, total, status = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int32(0)
+    st = lib().cat_workspace_report(ctypes.c_void_p(ws.data_ptr()), _stream(), ctypes.byref(last),
+                                    ctypes.byref(total), ctypes.byref(status))
+    _check(st, "cat_workspace_report")
+    return dict(refined_rows_last=last.value, refined_rows_total=total.value, device_status=status.value)
 
 
 def cat_version() -> str:

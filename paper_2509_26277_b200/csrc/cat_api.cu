@@ -310,6 +310,20 @@ cat_status_t cat_solve_gamma_beta(const double *sumQ, const double *sumF, const 
     return CAT_OK;
 }
 
+cat_status_t cat_workspace_report(const void *workspace, void *stream, int64_t *refined_last_host,
+                                  int64_t *refined_total_host, int32_t *device_status_host)
+{
+    if (!workspace) return CAT_ERR_NULL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    Control h{};
+    CAT_CUDA(cudaMemcpyAsync(&h, workspace, sizeof(Control), cudaMemcpyDeviceToHost, s));
+    CAT_CUDA(cudaStreamSynchronize(s));
+    if (refined_last_host) *refined_last_host = h.refined_last;
+    if (refined_total_host) *refined_total_host = h.refined_total;
+    if (device_status_host) *device_status_host = h.device_status;
+    return CAT_OK;
+}
+
 const char *cat_status_string(cat_status_t status)
 {
     switch (status) {

@@ -411,8 +411,11 @@ cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *
 // exact decision for queued rows
 // ======================================================================================
 
-constexpr int R_THREADS = 128;
+constexpr int R_THREADS = 256;
+constexpr int R_WARPS = R_THREADS / 32;
 
+// One CTA per queued row: warp w evaluates centroids w, w + 8, ... in direct form with fp64
+// accumulation; the CTA then takes the smallest distance, lowest index on equality.
 template <bool AFFINE>
 __global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restrict__ Y, int64_t N,
                                                            int D, int K, const float *__restrict__ C,
@@ -421,6 +424,9 @@ __global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restri
                                                            Control *ctl, const float *gamma,
                                                            const float *beta, float *out)
 {
+    __shared__ double s_best[R_WARPS];
+    __shared__ int s_idx[R_WARPS];
+    __shared__ int s_label;
     int count = ctl->refine_count;
     if ((int64_t)count > N) count = (int)N;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -428,35 +434,65 @@ __global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restri
         ctl->refined_last = count;
     }
     const int lane = threadIdx.x & 31;
-    const int warps_per_block = R_THREADS / 32;
-    const int gw = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-    const int nw = gridDim.x * warps_per_block;
-    for (int it = gw; it < count; it += nw) {
+    const int w = threadIdx.x >> 5;
+    for (int it = blockIdx.x; it < count; it += gridDim.x) {
         int64_t row = refine_rows[it];
-        if (row < 0 || row >= N) continue;
+        if (row < 0 || row >= N) continue;  // uniform across the CTA
         const float *y = Y + (size_t)row * D;
         double best = CUDART_INF;
-        int bk = 0;
-        for (int k = 0; k < K; ++k) {
+        int bk = K;  // "none": loses every comparison below
+        for (int k = w; k < K; k += R_WARPS) {
             const float *c = C + (size_t)k * D;
-            double s = 0.0;
-            for (int j = lane; j < D; j += 32) {
-                double d = (double)y[j] - (double)c[j];
-                s = fma(d, d, s);
+            double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+            int j = lane;
+            for (; j + 96 < D; j += 128) {
+                double d0 = (double)y[j] - (double)c[j];
+                double d1 = (double)y[j + 32] - (double)c[j + 32];
+                double d2 = (double)y[j + 64] - (double)c[j + 64];
+                double d3 = (double)y[j + 96] - (double)c[j + 96];
+                s0 = fma(d0, d0, s0);
+                s1 = fma(d1, d1, s1);
+                s2 = fma(d2, d2, s2);
+                s3 = fma(d3, d3, s3);
             }
-            s = warp_sum(s);
+            for (; j < D; j += 32) {
+                double d0 = (double)y[j] - (double)c[j];
+                s0 = fma(d0, d0, s0);
+            }
+            double s = warp_sum((s0 + s1) + (s2 + s3));
             if (s < best) {
                 best = s;
                 bk = k;
             }
         }
-        if (lane == 0) labels[row] = bk;
-        if (AFFINE) {
-            const float *g = gamma + (size_t)bk * D;
-            const float *b = beta + (size_t)bk * D;
-            float *o = out + (size_t)row * D;
-            for (int j = lane; j < D; j += 32) o[j] = fmaf(g[j], y[j], b[j]);
+        if (lane == 0) {
+            s_best[w] = best;
+            s_idx[w] = bk;
         }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double b = s_best[0];
+            int k = s_idx[0];
+#pragma unroll
+            for (int q = 1; q < R_WARPS; ++q) {
+                if (s_best[q] < b || (s_best[q] == b && s_idx[q] < k)) {
+                    b = s_best[q];
+                    k = s_idx[q];
+                }
+            }
+            if (k >= K) k = 0;  // only when every distance is NaN
+            labels[row] = k;
+            s_label = k;
+        }
+        __syncthreads();
+        if (AFFINE) {
+            const int l = s_label;
+            const float *g = gamma + (size_t)l * D;
+            const float *bb = beta + (size_t)l * D;
+            float *o = out + (size_t)row * D;
+            for (int j = threadIdx.x; j < D; j += R_THREADS) o[j] = fmaf(g[j], y[j], bb[j]);
+        }
+        __syncthreads();
     }
 }
 
@@ -464,8 +500,7 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
                           int32_t *labels, const int32_t *refine_rows, Control *ctl,
                           const float *gamma, const float *beta, float *out, cudaStream_t s)
 {
-    int64_t want = (N + (R_THREADS / 32) - 1) / (R_THREADS / 32);
-    int blocks = (int)(want < 592 ? want : 592);
+    int blocks = (int)(N < 1184 ? N : 1184);
     if (out)
         refine_kernel<true><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
                                                          gamma, beta, out);

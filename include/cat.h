@@ -129,6 +129,34 @@ cat_status_t cat_assign(const float *Yq, int64_t N, int32_t D, int32_t K,
                         const float *centroids, int32_t *labels_out,
                         void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * cat_assign without any workspace: the same labels as cat_assign, for callers that
+ * cannot allocate device memory.  (The paper has no counterpart: this is a packaging
+ * variant of the assignment step, not a step of the method.)
+ *
+ * Who needs it: code that runs where a device allocation is impossible or unwelcome --
+ * a serving loop that must never hit the allocator (cudaMalloc may synchronise the whole
+ * device), a plug-in that only ever receives its input and output buffers from a host
+ * framework that owns all device memory, or a process whose memory budget was fixed at
+ * start-up.  Such callers cannot provide the scratch cat_assign asks for, so this entry
+ * point keeps its own: a fixed array inside the library image, about 1 MiB per GPU that
+ * loads the library, held until the process exits.
+ *
+ *   - Limits: N <= CAT_NOALLOC_MAX_ROWS, K <= CAT_MAX_K, D <= CAT_MAX_D; anything larger
+ *     returns CAT_ERR_UNSUPPORTED ("size beyond the supported limits") and enqueues nothing.
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current); make that first call outside any
+ *     stream capture.  Later calls only launch kernels on `stream`.
+ *   - All calls on one device share the one array.  Calls that may overlap on the GPU
+ *     (different streams without ordering between them, or different host threads) race on
+ *     it and give wrong labels; order them on one stream or with events.  The array keeps
+ *     the previous call's contents; the call itself clears what has to start at zero.
+ */
+#define CAT_NOALLOC_MAX_ROWS 262144
+cat_status_t cat_assign_noalloc(const float *Yq, int64_t N, int32_t D, int32_t K,
+                                const float *centroids, int32_t *labels_out, void *stream);
+
 /* Per-cluster column sums of Y (fp64) and cluster sizes for given labels:
  * sums_out [K, D] double, counts_out [K] int64.  Labels must lie in [0, K).
  * Rows are added in a fixed order: results are reproducible run to run.

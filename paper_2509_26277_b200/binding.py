@@ -26,7 +26,8 @@ MAX_D = 16384
 
 EXPORTS = [
     "cat_fit_workspace_bytes", "cat_fit", "cat_fit_from", "cat_apply_workspace_bytes",
-    "cat_apply", "cat_apply_blend", "cat_assign", "cat_cluster_sums", "cat_centroids_from_sums",
+    "cat_apply", "cat_apply_blend", "cat_assign", "cat_assign_noalloc", "cat_cluster_sums",
+    "cat_centroids_from_sums",
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
     "cat_status_string",
@@ -78,6 +79,8 @@ def lib():
     L.cat_apply.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     L.cat_apply_blend.argtypes = [vp, i64, i32, i32, vp, vp, vp, f32, vp, vp, vp, sz, vp]
     L.cat_assign.argtypes = [vp, i64, i32, i32, vp, vp, vp, sz, vp]
+    L.cat_assign_noalloc.argtypes = [vp, i64, i32, i32, vp, vp, vp]
+    L.cat_assign_noalloc.restype = ctypes.c_int
     L.cat_cluster_sums.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, sz, vp]
     L.cat_centroids_from_sums.argtypes = [vp, vp, i32, i32, vp, vp]
     L.cat_centred_moments.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, vp, vp, sz, vp]
@@ -242,6 +245,22 @@ def cat_assign(Yq, centroids, ws=None):
                           ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream())
     _check(st, "cat_assign")
     return labels
+
+
+NOALLOC_MAX_ROWS = 262144
+
+
+def cat_assign_noalloc(Yq, centroids, labels_out):
+    """cat_assign_noalloc: labels into the caller's `labels_out`; the library uses its own
+    fixed scratch (no workspace, no allocation).  At most NOALLOC_MAX_ROWS rows; calls that
+    could overlap on the GPU must be ordered by the caller."""
+    N, D = Yq.shape
+    K = centroids.shape[0]
+    st = lib().cat_assign_noalloc(_dev(Yq, torch.float32, None, "Yq"), N, D, K,
+                                  _dev(centroids, torch.float32, (K, D), "centroids"),
+                                  _dev(labels_out, torch.int32, (N,), "labels_out"), _stream())
+    _check(st, "cat_assign_noalloc")
+    return labels_out
 
 
 def cat_cluster_sums(Y, labels, K: int, ws=None):

@@ -228,6 +228,14 @@ cat_status_t cat_fit_host(const float *Yq_host, const float *Yfp_host, int64_t N
 cat_status_t cat_workspace_report(const void *workspace, void *stream, int64_t *refined_last_host,
                                   int64_t *refined_total_host, int32_t *device_status_host);
 
+/* Kernel selection for the distance contraction.  With K >= min_k (and D % 4 == 0,
+ * K <= 256) the scores are formed on the tensor cores (tcgen05, TF32 operands, fp32
+ * accumulation); below it on the fp32 pipes.  Either way undecided rows are settled in
+ * fp64, so the labels are the same.  Default 32: for smaller K the contraction is not
+ * compute-limited.  Process-wide setting. */
+void cat_set_tensor_core_min_k(int32_t min_k);
+int32_t cat_get_tensor_core_min_k(void);
+
 const char *cat_status_string(cat_status_t status);
 int cat_last_cuda_error(void);           /* cudaError_t of the last failing runtime call on this thread */
 const char *cat_version(void);

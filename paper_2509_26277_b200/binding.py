@@ -30,7 +30,7 @@ EXPORTS = [
     "cat_centroids_from_sums",
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
-    "cat_status_string",
+    "cat_set_tensor_core_min_k", "cat_get_tensor_core_min_k", "cat_status_string",
     "cat_last_cuda_error", "cat_version", "cat_kernel_launches",
 ]
 
@@ -93,6 +93,9 @@ def lib():
         getattr(L, name).restype = ctypes.c_int
     L.cat_workspace_report.argtypes = [vp, vp, vp, vp, vp]
     L.cat_workspace_report.restype = ctypes.c_int
+    L.cat_set_tensor_core_min_k.argtypes = [i32]
+    L.cat_set_tensor_core_min_k.restype = None
+    L.cat_get_tensor_core_min_k.restype = i32
     L.cat_status_string.argtypes = [ctypes.c_int]
     L.cat_status_string.restype = ctypes.c_char_p
     L.cat_last_cuda_error.restype = ctypes.c_int
@@ -350,6 +353,14 @@ def cat_workspace_report(ws) -> dict:
                                     ctypes.byref(total), ctypes.byref(status))
     _check(st, "cat_workspace_report")
     return dict(refined_rows_last=last.value, refined_rows_total=total.value, device_status=status.value)
+
+
+def cat_set_tensor_core_min_k(min_k: int) -> None:
+    lib().cat_set_tensor_core_min_k(int(min_k))
+
+
+def cat_get_tensor_core_min_k() -> int:
+    return int(lib().cat_get_tensor_core_min_k())
 
 
 def cat_version() -> str:

@@ -35,6 +35,7 @@ static void carve_assign_into(Carver &c, AssignWs &w, int64_t N, int D, int K)
     w.labels = c.take<int32_t>((size_t)N);
     w.gamma_b = c.take<float>((size_t)K * D);
     w.beta_b = c.take<float>((size_t)K * D);
+    w.ynorm2 = c.take<float>((size_t)N);
 }
 
 AssignWs carve_assign(void *base, int64_t N, int D, int K)
@@ -82,13 +83,28 @@ static cat_status_t check_shape(int64_t N, int32_t D, int32_t K, bool need_n_ge_
         if (!cuda_ok((expr))) return CAT_ERR_CUDA;      \
     } while (0)
 
-// norms -> fast assignment -> exact pass for undecided rows
+static std::atomic<int> g_tc_min_k{32};
+
+static bool use_tensor_path(int64_t N, int D, int K)
+{
+    return K >= g_tc_min_k.load(std::memory_order_relaxed) && tc_supported(N, D, K);
+}
+
+// norms -> fast assignment (tensor cores for large K, fp32 pipes otherwise) -> exact pass for
+// undecided rows.  row_norms_ready: w.ynorm2 already holds this Y's squared row norms.
 static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const float *C,
                                int32_t *labels, const AssignWs &w, const float *gamma,
-                               const float *beta, float *out, cudaStream_t s)
+                               const float *beta, float *out, cudaStream_t s,
+                               bool row_norms_ready = false, bool top_level = true)
 {
-    CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s));
-    CAT_CUDA(launch_assign(Y, N, D, K, C, w.cnorm, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
+    CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s, top_level));
+    if (use_tensor_path(N, D, K)) {
+        if (!out && !row_norms_ready) CAT_CUDA(launch_row_norms(Y, N, D, w.ynorm2, s));
+        CAT_CUDA(launch_assign_tc(Y, N, D, K, C, w.cnorm, w.ynorm2, labels, w.refine_rows, w.ctl, gamma,
+                                  beta, out, s));
+    } else {
+        CAT_CUDA(launch_assign(Y, N, D, K, C, w.cnorm, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
+    }
     if (K > 1) CAT_CUDA(launch_refine(Y, N, D, K, C, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
     return CAT_OK;
 }
@@ -220,8 +236,10 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     CAT_CUDA(cudaMemcpyAsync(C, init_centroids ? init_centroids : Yq, KD * sizeof(float),
                              cudaMemcpyDeviceToDevice, s));
 
+    const bool tc = use_tensor_path(N, D, K);
+    if (tc) CAT_CUDA(launch_row_norms(Yq, N, D, w.a.ynorm2, s));   // Yq is fixed: once per fit
     for (int t = 0; t < iters; ++t) {
-        st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s);
+        st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false);
         if (st != CAT_OK) return st;
         st = run_cluster_sums(Yq, labels, N, D, K, w, w.sumQ, w.counts, s);
         if (st != CAT_OK) return st;
@@ -229,7 +247,7 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     }
 
     // final assignment, then the closed form
-    st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s);
+    st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false);
     if (st != CAT_OK) return st;
     st = run_cluster_sums(Yq, labels, N, D, K, w, w.sumQ, w.counts, s);
     if (st != CAT_OK) return st;
@@ -323,6 +341,13 @@ cat_status_t cat_workspace_report(const void *workspace, void *stream, int64_t *
     if (device_status_host) *device_status_host = h.device_status;
     return CAT_OK;
 }
+
+void cat_set_tensor_core_min_k(int32_t min_k)
+{
+    g_tc_min_k.store(min_k < 1 ? 1 : min_k, std::memory_order_relaxed);
+}
+
+int32_t cat_get_tensor_core_min_k(void) { return g_tc_min_k.load(std::memory_order_relaxed); }
 
 const char *cat_status_string(cat_status_t status)
 {

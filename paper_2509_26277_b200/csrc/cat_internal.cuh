@@ -54,6 +54,7 @@ struct AssignWs {          // what assign/apply need
     int32_t *labels;       // [N] (used when the caller passes no labels_out)
     float *gamma_b;        // [K*D] blended gamma (alpha != 1)
     float *beta_b;         // [K*D]
+    float *ynorm2;         // [N] squared row norms (tensor-core labels-only path)
     size_t bytes;
 };
 AssignWs carve_assign(void *base, int64_t N, int D, int K);
@@ -72,9 +73,10 @@ FitWs carve_fit(void *base, int64_t N, int D, int K);
 // ---------------------------------------------------------------- kernel launchers (cat_kernels.cu)
 // All return a cudaError_t from the launch; none synchronises.
 
-// cnorm[k] = ||c_k||^2 (fp64 accumulate, rounded to fp32); also resets ctl->refine_count.
+// cnorm[k] = ||c_k||^2 (fp64 accumulate, rounded up to fp32); also resets ctl->refine_count,
+// and with reset_all the status word and the counters (start of a top-level call).
 cudaError_t launch_centroid_norms(const float *C, int D, int K, float *cnorm, Control *ctl,
-                                  cudaStream_t s);
+                                  cudaStream_t s, bool reset_all = false);
 
 // Fast fp32 scores + certainty test; optional fused affine epilogue.
 cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *C,
@@ -85,6 +87,13 @@ cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *
 cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *C,
                           int32_t *labels, const int32_t *refine_rows, Control *ctl,
                           const float *gamma, const float *beta, float *out, cudaStream_t s);
+
+// Tensor-core (tcgen05, TF32) variant of launch_assign; ynorm2 is needed when out == nullptr.
+bool tc_supported(int64_t N, int D, int K);
+cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaStream_t s);
+cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,
+                             const float *ynorm2, int32_t *labels, int32_t *refine_rows, Control *ctl,
+                             const float *gamma, const float *beta, float *out, cudaStream_t s);
 
 // Segmented sums.  mode 0: partial[chunk][0] += Y rows per label (+ counts).
 // mode 1: centred moments: planes selected by mask (1 = var, 2 = cov).

@@ -55,11 +55,18 @@ __device__ __forceinline__ double warp_sum(double v)
 // ======================================================================================
 
 __global__ void centroid_norms_kernel(const float *__restrict__ C, int D, int K,
-                                      float *__restrict__ cnorm, Control *ctl)
+                                      float *__restrict__ cnorm, Control *ctl, int reset_all)
 {
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
-    if (blockIdx.x == 0 && threadIdx.x == 0) ctl->refine_count = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctl->refine_count = 0;
+        if (reset_all) {
+            ctl->device_status = CAT_OK;
+            ctl->refined_total = 0;
+            ctl->refined_last = 0;
+        }
+    }
     if (warp >= K) return;
     const float *c = C + (size_t)warp * D;
     double s = 0.0;
@@ -73,11 +80,11 @@ __global__ void centroid_norms_kernel(const float *__restrict__ C, int D, int K,
 }
 
 cudaError_t launch_centroid_norms(const float *C, int D, int K, float *cnorm, Control *ctl,
-                                  cudaStream_t s)
+                                  cudaStream_t s, bool reset_all)
 {
     int threads = 128;
     int blocks = (K * 32 + threads - 1) / threads;
-    centroid_norms_kernel<<<blocks, threads, 0, s>>>(C, D, K, cnorm, ctl);
+    centroid_norms_kernel<<<blocks, threads, 0, s>>>(C, D, K, cnorm, ctl, reset_all ? 1 : 0);
     count_launch();
     return cudaGetLastError();
 }

@@ -21,6 +21,16 @@ from tests.parity import close, labels_match
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["fp32", "tensor"], autouse=True)
+def contraction_path(request):
+    """Every case runs twice: distance contraction forced onto the fp32 pipes, and forced onto
+    the tensor cores wherever that path applies (D % 4 == 0, K <= 256)."""
+    old = B.cat_get_tensor_core_min_k()
+    B.cat_set_tensor_core_min_k(1 << 30 if request.param == "fp32" else 1)
+    yield request.param
+    B.cat_set_tensor_core_min_k(old)
+
+
 def dev(a):
     return torch.as_tensor(np.ascontiguousarray(a)).cuda()
 

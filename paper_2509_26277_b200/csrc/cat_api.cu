@@ -36,6 +36,8 @@ static void carve_assign_into(Carver &c, AssignWs &w, int64_t N, int D, int K)
     w.gamma_b = c.take<float>((size_t)K * D);
     w.beta_b = c.take<float>((size_t)K * D);
     w.ynorm2 = c.take<float>((size_t)N);
+    w.cand_rows = c.take<int32_t>((size_t)N);
+    w.cand_list = c.take<uint64_t>((size_t)N);
 }
 
 AssignWs carve_assign(void *base, int64_t N, int D, int K)
@@ -100,8 +102,10 @@ static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const fl
     CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s, top_level));
     if (use_tensor_path(N, D, K)) {
         if (!out && !row_norms_ready) CAT_CUDA(launch_row_norms(Y, N, D, w.ynorm2, s));
-        CAT_CUDA(launch_assign_tc(Y, N, D, K, C, w.cnorm, w.ynorm2, labels, w.refine_rows, w.ctl, gamma,
-                                  beta, out, s));
+        CAT_CUDA(launch_assign_tc(Y, N, D, K, C, w.cnorm, w.ynorm2, labels, w.refine_rows, w.cand_rows,
+                                  w.cand_list, w.ctl, gamma, beta, out, s));
+        CAT_CUDA(launch_refine_candidates(Y, N, D, K, C, labels, w.cand_rows, w.cand_list, w.ctl, gamma,
+                                          beta, out, s));
     } else {
         CAT_CUDA(launch_assign(Y, N, D, K, C, w.cnorm, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
     }

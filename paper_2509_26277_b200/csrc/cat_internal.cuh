@@ -30,8 +30,10 @@ struct Control {
     int32_t refine_count;        // rows queued for the exact fp64 pass by the current assignment
     int32_t device_status;       // CAT_OK or CAT_ERR_DEVICE_TIMEOUT
     int64_t refined_total;       // running total over assignments
-    int64_t refined_last;        // refine_count of the latest finished assignment
-    int64_t pad[5];
+    int64_t refined_last;        // rows of the latest finished assignment that took an exact pass
+    int32_t cand_count;          // rows queued with a short candidate list by the current assignment
+    int32_t pad0;
+    int64_t pad[4];
 };
 
 // Geometry of the segmented-sum kernels for one (N, D, K): identical in the
@@ -55,6 +57,8 @@ struct AssignWs {          // what assign/apply need
     float *gamma_b;        // [K*D] blended gamma (alpha != 1)
     float *beta_b;         // [K*D]
     float *ynorm2;         // [N] squared row norms (tensor-core labels-only path)
+    int32_t *cand_rows;    // [N] rows queued with candidates
+    uint64_t *cand_list;   // [N] their candidates, 4 x 16 bit
     size_t bytes;
 };
 AssignWs carve_assign(void *base, int64_t N, int D, int K);
@@ -92,8 +96,15 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
 bool tc_supported(int64_t N, int D, int K);
 cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaStream_t s);
 cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,
-                             const float *ynorm2, int32_t *labels, int32_t *refine_rows, Control *ctl,
+                             const float *ynorm2, int32_t *labels, int32_t *refine_rows,
+                             int32_t *cand_rows, uint64_t *cand_list, Control *ctl,
                              const float *gamma, const float *beta, float *out, cudaStream_t s);
+
+// Exact fp64 decision among the listed candidates of each queued row; optional affine output.
+cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, const float *C,
+                                     int32_t *labels, const int32_t *cand_rows,
+                                     const uint64_t *cand_list, Control *ctl, const float *gamma,
+                                     const float *beta, float *out, cudaStream_t s);
 
 // Segmented sums.  mode 0: partial[chunk][0] += Y rows per label (+ counts).
 // mode 1: centred moments: planes selected by mask (1 = var, 2 = cov).

@@ -61,6 +61,7 @@ __global__ void centroid_norms_kernel(const float *__restrict__ C, int D, int K,
     int lane = threadIdx.x & 31;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         ctl->refine_count = 0;
+        ctl->cand_count = 0;
         if (reset_all) {
             ctl->device_status = CAT_OK;
             ctl->refined_total = 0;
@@ -437,8 +438,9 @@ __global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restri
     int count = ctl->refine_count;
     if ((int64_t)count > N) count = (int)N;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
+        // the candidate pass (if any) ran before this kernel and has already added its rows
         ctl->refined_total += count;
-        ctl->refined_last = count;
+        ctl->refined_last = count + ctl->cand_count;
     }
     const int lane = threadIdx.x & 31;
     const int w = threadIdx.x >> 5;
@@ -514,6 +516,82 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
     else
         refine_kernel<false><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
                                                           gamma, beta, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// Exact decision among at most four listed candidates: one warp per queued row, the
+// candidates' fp64 direct-form distances formed together (the row is read once).
+constexpr int RC_THREADS = 256;
+
+template <bool AFFINE>
+__global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
+    const float *__restrict__ Y, int64_t N, int D, int K, const float *__restrict__ C, int32_t *labels,
+    const int32_t *__restrict__ cand_rows, const uint64_t *__restrict__ cand_list, Control *ctl,
+    const float *gamma, const float *beta, float *out)
+{
+    int count = ctl->cand_count;
+    if ((int64_t)count > N) count = (int)N;
+    if (blockIdx.x == 0 && threadIdx.x == 0) ctl->refined_total += count;
+    const int lane = threadIdx.x & 31;
+    const int gw = blockIdx.x * (RC_THREADS / 32) + (threadIdx.x >> 5);
+    const int nw = gridDim.x * (RC_THREADS / 32);
+    for (int it = gw; it < count; it += nw) {
+        const int64_t row = cand_rows[it];
+        const uint64_t packed = cand_list[it];
+        if (row < 0 || row >= N) continue;
+        int cand[4];
+        const float *cp[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int k = (int)((packed >> (16 * q)) & 0xFFFFu);
+            cand[q] = (k < K) ? k : -1;
+            cp[q] = C + (size_t)(k < K ? k : 0) * D;
+        }
+        const float *y = Y + (size_t)row * D;
+        double s[4] = {0.0, 0.0, 0.0, 0.0};
+        for (int j = lane; j < D; j += 32) {
+            const double yv = (double)y[j];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const double d = yv - (double)cp[q][j];
+                s[q] = fma(d, d, s[q]);
+            }
+        }
+        double best = CUDART_INF;
+        int bk = K;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const double v = warp_sum(s[q]);
+            if (cand[q] >= 0 && (v < best || (v == best && cand[q] < bk))) {
+                best = v;
+                bk = cand[q];
+            }
+        }
+        if (bk >= K) bk = (cand[0] >= 0) ? cand[0] : 0;   // only when every distance is NaN
+        if (lane == 0) labels[row] = bk;
+        if (AFFINE) {
+            const float *g = gamma + (size_t)bk * D;
+            const float *bb = beta + (size_t)bk * D;
+            float *o = out + (size_t)row * D;
+            for (int j = lane; j < D; j += 32) o[j] = fmaf(g[j], y[j], bb[j]);
+        }
+    }
+}
+
+cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, const float *C,
+                                     int32_t *labels, const int32_t *cand_rows,
+                                     const uint64_t *cand_list, Control *ctl, const float *gamma,
+                                     const float *beta, float *out, cudaStream_t s)
+{
+    int64_t want = (N + (RC_THREADS / 32) - 1) / (RC_THREADS / 32);
+    int blocks = (int)(want < 1184 ? want : 1184);
+    if (out)
+        refine_candidates_kernel<true><<<blocks, RC_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows,
+                                                                    cand_list, ctl, gamma, beta, out);
+    else
+        refine_candidates_kernel<false><<<blocks, RC_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows,
+                                                                     cand_list, ctl, gamma, beta, out);
     count_launch();
     return cudaGetLastError();
 }

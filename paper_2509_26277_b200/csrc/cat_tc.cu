@@ -171,6 +171,8 @@ struct TcParams {
     const float *ynorm2;   // [N] squared row norms (labels-only mode)
     int32_t *labels;
     int32_t *refine_rows;
+    int32_t *cand_rows;    // rows whose exact decision only needs the listed candidates
+    uint64_t *cand_list;   // four 16-bit centroid indices per entry (0xFFFF = unused)
     Control *ctl;
     const float *gamma;
     const float *beta;
@@ -194,9 +196,8 @@ struct TcShared {
     int abort_flag;
     float red[16];
     float cn[256];
-    float best[2][TC_BM];
-    float second[2][TC_BM];
-    int idx[2][TC_BM];
+    float4 top_score[2][TC_BM];   // four smallest scores of each row, ascending
+    int4 top_idx[2][TC_BM];       // their centroid indices
 };
 
 __device__ __forceinline__ float tc_error_bound(int D, float ysq, float cmax2)
@@ -204,6 +205,28 @@ __device__ __forceinline__ float tc_error_bound(int D, float ysq, float cmax2)
     const float u = 5.9604645e-8f;   // 2^-24
     const float a = 3.90625e-3f + (2.f * (float)D + 2.f) * 2.3841858e-7f;  // 2^-8 + (2D+2) 2^-22
     return 1.0625f * (a * sqrtf(ysq) * sqrtf(cmax2) + 4.f * u * cmax2);
+}
+
+// Decision for one row from its four smallest scores.  Returns true when the fast argmin is
+// certainly exact.  Otherwise the row is queued: with the centroids whose score lies within
+// 2e of the best when those are known to be among the four, else for a scan of all K.
+__device__ __forceinline__ bool tc_decide(const TcParams &p, int64_t row, float4 sc, int4 id, float e)
+{
+    const float lim = 2.f * e;
+    if (p.K == 1 || (sc.y - sc.x) > lim) return true;
+    const bool more = !((sc.w - sc.x) > lim);   // the 4th is a candidate too (or NaN): others may be
+    if (more && p.K > 4) {
+        int slot = atomicAdd(&p.ctl->refine_count, 1);
+        p.refine_rows[slot] = (int32_t)row;
+    } else {
+        uint64_t c = (uint64_t)(uint16_t)id.x | ((uint64_t)(uint16_t)id.y << 16);
+        c |= (uint64_t)(((sc.z - sc.x) > lim || p.K < 3) ? 0xFFFFu : (uint16_t)id.z) << 32;
+        c |= (uint64_t)(((sc.w - sc.x) > lim || p.K < 4) ? 0xFFFFu : (uint16_t)id.w) << 48;
+        int slot = atomicAdd(&p.ctl->cand_count, 1);
+        p.cand_rows[slot] = (int32_t)row;
+        p.cand_list[slot] = c;
+    }
+    return false;
 }
 
 template <bool AFFINE>
@@ -331,21 +354,25 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             if (scorer) {
                 if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
                 tc_fence_after();
-                float b1 = CUDART_INF_F, b2 = CUDART_INF_F;
-                int bi = 0;
+                float b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F, b4 = CUDART_INF_F;
+                int i1 = 0, i2 = 0, i3 = 0, i4 = 0;
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
                 for (int c = 0; c < p.npad; c += 16) {
                     float v[16];
                     tmem_ld16(taddr + (uint32_t)c, v);
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        float sc = fmaf(-2.f, v[j], sh.cn[c + j]);
-                        if (sc < b1) {
-                            b2 = b1;
-                            b1 = sc;
-                            bi = c + j;
-                        } else if (sc < b2) {
-                            b2 = sc;
+                        const float sc = fmaf(-2.f, v[j], sh.cn[c + j]);
+                        if (sc < b4) {
+                            const int n = c + j;
+                            if (sc < b3) {
+                                b4 = b3; i4 = i3;
+                                if (sc < b2) {
+                                    b3 = b2; i3 = i2;
+                                    if (sc < b1) { b2 = b1; i2 = i1; b1 = sc; i1 = n; }
+                                    else { b2 = sc; i2 = n; }
+                                } else { b3 = sc; i3 = n; }
+                            } else { b4 = sc; i4 = n; }
                         }
                     }
                 }
@@ -356,21 +383,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 const int r = quarter * 32 + lane;
                 if (AFFINE) {
                     if (!mbar_wait_warp(smem_u32(&sh.lab_empty[b]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
-                    sh.best[b][r] = b1;
-                    sh.second[b][r] = b2;
-                    sh.idx[b][r] = bi;
+                    sh.top_score[b][r] = make_float4(b1, b2, b3, b4);
+                    sh.top_idx[b][r] = make_int4(i1, i2, i3, i4);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&sh.lab_full[b]));
                 } else {
                     const int64_t row = row0 + r;
                     if (row < p.N) {
-                        float e = tc_error_bound(p.D, p.ynorm2[row], cmax2);
-                        bool certain = (p.K == 1) || ((b2 - b1) > 2.f * e);
-                        p.labels[row] = bi;
-                        if (!certain) {
-                            int slot = atomicAdd(&p.ctl->refine_count, 1);
-                            p.refine_rows[slot] = (int32_t)row;
-                        }
+                        const float e = tc_error_bound(p.D, p.ynorm2[row], cmax2);
+                        p.labels[row] = i1;
+                        tc_decide(p, row, make_float4(b1, b2, b3, b4), make_int4(i1, i2, i3, i4), e);
                     }
                 }
             }
@@ -384,8 +406,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 for (int r = ew; r < TC_BM; r += NEPI) {
                     const int64_t row = row0 + r;
                     if (row >= p.N) break;
-                    const int l = sh.idx[b][r];
-                    const float gap = sh.second[b][r] - sh.best[b][r];
+                    const float4 tsc = sh.top_score[b][r];
+                    const int4 tid4 = sh.top_idx[b][r];
+                    const int l = tid4.x;
                     const float4 *y4 = Y4 + (size_t)row * D4;
                     const float4 *g4 = G4 + (size_t)l * D4;
                     const float4 *b4 = B4 + (size_t)l * D4;
@@ -412,7 +435,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         }
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
-                        const bool certain = (p.K == 1) || (gap > 2.f * tc_error_bound(p.D, ysq, cmax2));
+                        const float e = tc_error_bound(p.D, ysq, cmax2);
+                        const bool certain = (p.K == 1) || ((tsc.y - tsc.x) > 2.f * e);
                         if (certain) {
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {
@@ -422,10 +446,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         }
                         if (lane == 0) {
                             p.labels[row] = l;
-                            if (!certain) {
-                                int slot = atomicAdd(&p.ctl->refine_count, 1);
-                                p.refine_rows[slot] = (int32_t)row;
-                            }
+                            if (!certain) tc_decide(p, row, tsc, tid4, e);
                         }
                     } else {
                         float ysq = 0.f;
@@ -438,7 +459,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         }
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
-                        const bool certain = (p.K == 1) || (gap > 2.f * tc_error_bound(p.D, ysq, cmax2));
+                        const float e = tc_error_bound(p.D, ysq, cmax2);
+                        const bool certain = (p.K == 1) || ((tsc.y - tsc.x) > 2.f * e);
                         if (certain) {
                             for (int c = lane; c < D4; c += 32) {
                                 float4 y = __ldcs(y4 + c);
@@ -454,10 +476,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         }
                         if (lane == 0) {
                             p.labels[row] = l;
-                            if (!certain) {
-                                int slot = atomicAdd(&p.ctl->refine_count, 1);
-                                p.refine_rows[slot] = (int32_t)row;
-                            }
+                            if (!certain) tc_decide(p, row, tsc, tid4, e);
                         }
                     }
                 }
@@ -565,7 +584,8 @@ cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaS
 }
 
 cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,
-                             const float *ynorm2, int32_t *labels, int32_t *refine_rows, Control *ctl,
+                             const float *ynorm2, int32_t *labels, int32_t *refine_rows,
+                             int32_t *cand_rows, uint64_t *cand_list, Control *ctl,
                              const float *gamma, const float *beta, float *out, cudaStream_t s)
 {
     TcParams p{};
@@ -574,6 +594,8 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     p.ynorm2 = ynorm2;
     p.labels = labels;
     p.refine_rows = refine_rows;
+    p.cand_rows = cand_rows;
+    p.cand_list = cand_list;
     p.ctl = ctl;
     p.gamma = gamma;
     p.beta = beta;

@@ -54,12 +54,13 @@ FitWs carve_fit(void *base, int64_t N, int D, int K)
     Carver c(base);
     FitWs w{};
     carve_assign_into(c, w.a, N, D, K);
-    SumGeom g1 = sum_geometry(N, D, K, 1);
-    SumGeom g2 = sum_geometry(N, D, K, 2);
-    int nch = g1.nchunks > g2.nchunks ? g1.nchunks : g2.nchunks;
+    SegGeom g = seg_geometry(N, D, K);
     size_t KD = (size_t)K * D;
-    w.partial = c.take<double>((size_t)nch * 2 * KD);
-    w.partial_cnt = c.take<int32_t>((size_t)nch * K);
+    w.blk_hist = c.take<uint32_t>((size_t)g.nblk * K);
+    w.cluster_start = c.take<int32_t>((size_t)K + 1);
+    w.seg_start = c.take<int32_t>((size_t)K + 1);
+    w.order = c.take<int32_t>((size_t)N);
+    w.segpart = c.take<double>((size_t)g.max_segs * 2 * D);
     w.sumQ = c.take<double>(KD);
     w.sumF = c.take<double>(KD);
     w.var = c.take<double>(KD);
@@ -113,35 +114,34 @@ static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const fl
     return CAT_OK;
 }
 
-// per-cluster column sums of M (+ counts) into sums / counts
-static cat_status_t run_cluster_sums(const float *M, const int32_t *labels, int64_t N, int D, int K,
-                                     const FitWs &w, double *sums, int64_t *counts, cudaStream_t s)
+// sort the rows by label: counts, cluster/segment tables and `order` in the workspace
+static cat_status_t run_sort(const int32_t *labels, int64_t N, int D, int K, const FitWs &w,
+                             int64_t *counts, cudaStream_t s)
 {
-    SumGeom g = sum_geometry(N, D, K, 1);
-    CAT_CUDA(launch_cluster_partial(M, nullptr, labels, N, D, K, g, nullptr, nullptr, 0, w.partial,
-                                    w.partial_cnt, s));
-    CAT_CUDA(launch_reduce_partials(w.partial, w.partial_cnt, g.nchunks, 2, 0, D, K, sums, counts, s));
+    SegGeom g = seg_geometry(N, D, K);
+    CAT_CUDA(launch_label_sort(labels, N, K, g, w.blk_hist, counts, w.cluster_start, w.seg_start, w.order, s));
     return CAT_OK;
 }
 
-static cat_status_t run_centred(const float *Yq, const float *Yfp, const int32_t *labels, int64_t N,
-                                int D, int K, const FitWs &w, const double *meanQ,
-                                const double *meanF, double *var, double *cov, cudaStream_t s)
+// per-cluster column sums of M for the sorted rows; optionally the centroid update
+static cat_status_t run_sums(const float *M, int64_t N, int D, int K, const FitWs &w, const int64_t *counts,
+                             double *sums, float *C, cudaStream_t s)
 {
-    SumGeom g = sum_geometry(N, D, K, 2);
-    if (g.nacc == 2) {
-        CAT_CUDA(launch_cluster_partial(Yq, Yfp, labels, N, D, K, g, meanQ, meanF, 3, w.partial,
-                                        w.partial_cnt, s));
-        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 0, D, K, var, nullptr, s));
-        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 1, D, K, cov, nullptr, s));
-    } else {
-        CAT_CUDA(launch_cluster_partial(Yq, Yfp, labels, N, D, K, g, meanQ, meanF, 1, w.partial,
-                                        w.partial_cnt, s));
-        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 0, D, K, var, nullptr, s));
-        CAT_CUDA(launch_cluster_partial(Yq, Yfp, labels, N, D, K, g, meanQ, meanF, 2, w.partial,
-                                        w.partial_cnt, s));
-        CAT_CUDA(launch_reduce_partials(w.partial, nullptr, g.nchunks, 2, 1, D, K, cov, nullptr, s));
-    }
+    SegGeom g = seg_geometry(N, D, K);
+    CAT_CUDA(launch_segment_sums(0, M, nullptr, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D, K,
+                                 g, w.segpart, s));
+    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, counts, D, K, sums, nullptr, C, s));
+    return CAT_OK;
+}
+
+static cat_status_t run_centred(const float *Yq, const float *Yfp, int64_t N, int D, int K, const FitWs &w,
+                                const double *meanQ, const double *meanF, double *var, double *cov,
+                                cudaStream_t s)
+{
+    SegGeom g = seg_geometry(N, D, K);
+    CAT_CUDA(launch_segment_sums(2, Yq, Yfp, w.order, w.cluster_start, w.seg_start, meanQ, meanF, D, K, g,
+                                 w.segpart, s));
+    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, nullptr, D, K, var, cov, nullptr, s));
     return CAT_OK;
 }
 
@@ -245,21 +245,26 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     for (int t = 0; t < iters; ++t) {
         st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false);
         if (st != CAT_OK) return st;
-        st = run_cluster_sums(Yq, labels, N, D, K, w, w.sumQ, w.counts, s);
+        st = run_sort(labels, N, D, K, w, w.counts, s);
         if (st != CAT_OK) return st;
-        CAT_CUDA(launch_centroids_from_sums(w.sumQ, w.counts, D, K, C, s));
+        st = run_sums(Yq, N, D, K, w, w.counts, w.sumQ, C, s);   // sums -> centroid update
+        if (st != CAT_OK) return st;
     }
 
     // final assignment, then the closed form
     st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false);
     if (st != CAT_OK) return st;
-    st = run_cluster_sums(Yq, labels, N, D, K, w, w.sumQ, w.counts, s);
+    st = run_sort(labels, N, D, K, w, w.counts, s);
     if (st != CAT_OK) return st;
-    st = run_cluster_sums(Yfp, labels, N, D, K, w, w.sumF, w.counts, s);
-    if (st != CAT_OK) return st;
+    {
+        SegGeom g = seg_geometry(N, D, K);
+        CAT_CUDA(launch_segment_sums(1, Yq, Yfp, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D,
+                                     K, g, w.segpart, s));
+        CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, w.sumQ, w.sumF, nullptr, s));
+    }
     CAT_CUDA(launch_means_from_sums(w.sumQ, w.counts, D, K, meanQ, s));
     CAT_CUDA(launch_means_from_sums(w.sumF, w.counts, D, K, meanF, s));
-    st = run_centred(Yq, Yfp, labels, N, D, K, w, meanQ, meanF, w.var, w.cov, s);
+    st = run_centred(Yq, Yfp, N, D, K, w, meanQ, meanF, w.var, w.cov, s);
     if (st != CAT_OK) return st;
     CAT_CUDA(launch_solve(w.sumQ, w.sumF, w.var, w.cov, w.counts, D, K, gamma_out, beta_out, s));
     if (diag) CAT_CUDA(launch_fit_diag(w.a.ctl, w.counts, K, diag, s));
@@ -286,8 +291,10 @@ cat_status_t cat_cluster_sums(const float *Y, const int32_t *labels, int64_t N, 
     if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
         return CAT_ERR_WORKSPACE;
     FitWs w = carve_fit(workspace, N, D, K);
-    return run_cluster_sums(Y, labels, N, D, K, w, sums_out, counts_out,
-                            reinterpret_cast<cudaStream_t>(stream));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    st = run_sort(labels, N, D, K, w, counts_out, s);
+    if (st != CAT_OK) return st;
+    return run_sums(Y, N, D, K, w, counts_out, sums_out, nullptr, s);
 }
 
 cat_status_t cat_centroids_from_sums(const double *sums, const int64_t *counts, int32_t D,
@@ -315,8 +322,10 @@ cat_status_t cat_centred_moments(const float *Yq, const float *Yfp, const int32_
     if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
         return CAT_ERR_WORKSPACE;
     FitWs w = carve_fit(workspace, N, D, K);
-    return run_centred(Yq, Yfp, labels, N, D, K, w, meanQ, meanF, var_out, cov_out,
-                       reinterpret_cast<cudaStream_t>(stream));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    st = run_sort(labels, N, D, K, w, w.counts, s);
+    if (st != CAT_OK) return st;
+    return run_centred(Yq, Yfp, N, D, K, w, meanQ, meanF, var_out, cov_out, s);
 }
 
 cat_status_t cat_solve_gamma_beta(const double *sumQ, const double *sumF, const double *var_sum,

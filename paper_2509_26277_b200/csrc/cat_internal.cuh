@@ -36,18 +36,14 @@ struct Control {
     int64_t pad[4];
 };
 
-// Geometry of the segmented-sum kernels for one (N, D, K): identical in the
-// workspace query and at launch time.
-struct SumGeom {
-    int cpl;        // columns per lane: 1, 2 or 4 (slice width = 32*cpl)
-    int nacc;       // accumulator planes held in shared memory at once (1 or 2)
-    int copies;     // accumulator copies per cluster (spreads small K over the warps)
-    int nslices;    // column slices
-    int nchunks;    // row chunks
-    int64_t rows_per_chunk;
-    size_t smem_bytes;
+// Geometry of the sort-based segmented sums for one (N, D, K): identical in the workspace
+// query and at launch time.
+struct SegGeom {
+    int nblk;       // 1024-row blocks of the label sort
+    int seg_rows;   // rows per segment (multiple of 128)
+    int max_segs;   // upper bound on the number of segments: ceil(N / seg_rows) + K
 };
-SumGeom sum_geometry(int64_t N, int D, int K, int planes);
+SegGeom seg_geometry(int64_t N, int D, int K);
 
 struct AssignWs {          // what assign/apply need
     Control *ctl;
@@ -65,8 +61,11 @@ AssignWs carve_assign(void *base, int64_t N, int D, int K);
 
 struct FitWs {
     AssignWs a;
-    double *partial;       // [nchunks][2][K*D] partial sums of the segmented kernels
-    int32_t *partial_cnt;  // [nchunks][K]
+    uint32_t *blk_hist;    // [nblk][K] label histogram / offsets of the sort
+    int32_t *cluster_start; // [K+1] first position of each cluster in `order`
+    int32_t *seg_start;    // [K+1] first segment of each cluster
+    int32_t *order;        // [N] row indices sorted by label (stable)
+    double *segpart;       // [max_segs][2][D] per-segment partial sums
     double *sumQ, *sumF, *var, *cov;   // [K*D] each
     double *meanQ, *meanF;             // [K*D] each
     int64_t *counts;       // [K]
@@ -106,17 +105,23 @@ cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, co
                                      const uint64_t *cand_list, Control *ctl, const float *gamma,
                                      const float *beta, float *out, cudaStream_t s);
 
-// Segmented sums.  mode 0: partial[chunk][0] += Y rows per label (+ counts).
-// mode 1: centred moments: planes selected by mask (1 = var, 2 = cov).
-cudaError_t launch_cluster_partial(const float *Y, const float *F, const int32_t *labels,
-                                   int64_t N, int D, int K, const SumGeom &g,
-                                   const double *meanQ, const double *meanF, int mask,
-                                   double *partial, int32_t *partial_cnt, cudaStream_t s);
+// Stable sort of the row indices by label: counts[K], cluster_start[K+1], seg_start[K+1], order[N].
+// Labels outside [0, K) are left out.
+cudaError_t launch_label_sort(const int32_t *labels, int64_t N, int K, const SegGeom &g, uint32_t *blk_hist,
+                              int64_t *counts, int32_t *cluster_start, int32_t *seg_start, int32_t *order,
+                              cudaStream_t s);
 
-// out[k*D+j] = sum over chunks of partial[chunk][plane][k*D+j]; counts likewise (may be NULL).
-cudaError_t launch_reduce_partials(const double *partial, const int32_t *partial_cnt, int nchunks,
-                                   int nplanes, int plane, int D, int K, double *out,
-                                   int64_t *counts, cudaStream_t s);
+// Per-segment partial sums.  mode 0: column sums of Yq (plane 0); mode 1: of Yq and Yf (planes 0, 1);
+// mode 2: centred moments sum (q-muQ)^2 (plane 0) and sum (q-muQ)(f-muF) (plane 1).
+cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, const int32_t *order,
+                                const int32_t *cluster_start, const int32_t *seg_start, const double *meanQ,
+                                const double *meanF, int D, int K, const SegGeom &g, double *part,
+                                cudaStream_t s);
+
+// Adds each cluster's segment partials in order into out0 (and out1 if not NULL); with C also
+// writes the centroid float(out0 / n_k) for clusters with n_k > 0.
+cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
+                                   int K, double *out0, double *out1, float *C, cudaStream_t s);
 
 cudaError_t launch_centroids_from_sums(const double *sums, const int64_t *counts, int D, int K,
                                        float *C, cudaStream_t s);

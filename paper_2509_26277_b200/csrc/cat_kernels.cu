@@ -5,8 +5,6 @@
 //                           (+ fused per-cluster affine epilogue for inference)
 //   refine_kernel           exact fp64 direct-form decision for the rows the fast
 //                           scores cannot separate
-//   cluster_partial_kernel  segmented (per-cluster) column sums / centred moments with
-//                           block-private fp64 accumulators in shared memory
 //   small element-wise kernels for centroid update, means and the gamma/beta solve
 //
 // Label decision rule.  The K-Means assignment step needs argmin_k ||y - c_k||^2
@@ -597,280 +595,8 @@ cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, co
 }
 
 // ======================================================================================
-// segmented sums with block-private accumulators
-// ======================================================================================
-
-constexpr int S_THREADS = 512;
-constexpr int S_WARPS = S_THREADS / 32;
-constexpr int S_LABELS = 2048;               // labels staged per batch
-constexpr size_t S_ACC_BUDGET = 160 * 1024;  // bytes of shared memory for accumulators
-
-SumGeom sum_geometry(int64_t N, int D, int K, int planes)
-{
-    SumGeom g{};
-    g.copies = (K >= 4 * S_WARPS) ? 1 : (4 * S_WARPS + K - 1) / K;
-    const size_t kg = (size_t)K * g.copies;
-    g.nacc = planes;
-    g.cpl = 0;
-    for (int pass = 0; pass < 2 && g.cpl == 0; ++pass) {
-        for (int cpl = 4; cpl >= 1; cpl >>= 1) {
-            if (D % cpl) continue;
-            if (kg * 32 * cpl * sizeof(double) * g.nacc <= S_ACC_BUDGET) {
-                g.cpl = cpl;
-                break;
-            }
-        }
-        if (g.cpl == 0) g.nacc = 1;  // one plane at a time
-    }
-    if (g.cpl == 0) g.cpl = 1;  // unreachable for K <= CAT_MAX_K
-    const int sw = 32 * g.cpl;
-    g.nslices = (D + sw - 1) / sw;
-    int64_t maxchunks = (N + 255) / 256;
-    int64_t want = (296 + g.nslices - 1) / g.nslices;
-    int64_t nch = want < 1 ? 1 : want;
-    if (nch > 32) nch = 32;
-    if (nch > maxchunks) nch = maxchunks;
-    if (nch < 1) nch = 1;
-    g.nchunks = (int)nch;
-    g.rows_per_chunk = (N + nch - 1) / nch;
-    g.smem_bytes = kg * sw * sizeof(double) * g.nacc + kg * sizeof(int) + S_LABELS * sizeof(int);
-    return g;
-}
-
-struct SumParams {
-    const float *Y;
-    const float *F;
-    const int32_t *labels;
-    const double *meanQ;
-    const double *meanF;
-    double *partial;
-    int32_t *partial_cnt;
-    int64_t N;
-    int64_t rows_per_chunk;
-    int D;
-    int K;
-    int copies;
-    int mask;
-};
-
-template <int CPL>
-__device__ __forceinline__ void load_cols(const float *src, float (&v)[CPL])
-{
-    if constexpr (CPL == 4) {
-        float4 t = __ldg(reinterpret_cast<const float4 *>(src));
-        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-    } else if constexpr (CPL == 2) {
-        float2 t = __ldg(reinterpret_cast<const float2 *>(src));
-        v[0] = t.x; v[1] = t.y;
-    } else {
-        v[0] = __ldg(src);
-    }
-}
-
-// One CTA = (column slice, row chunk).  Warp w owns the accumulator rows v with
-// v % S_WARPS == w, where v = label * copies + row % copies, so no two warps ever touch
-// the same accumulator and every sum is formed in ascending row order.
-template <int CPL, int NACC, bool CENTRED>
-__global__ void __launch_bounds__(S_THREADS) cluster_partial_kernel(SumParams p)
-{
-    constexpr int SW = 32 * CPL;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int KG = p.K * p.copies;
-    double *acc = reinterpret_cast<double *>(smem_raw);               // [NACC][KG][SW]
-    int *cnt = reinterpret_cast<int *>(acc + (size_t)NACC * KG * SW);  // [KG]
-    int *lab_s = cnt + KG;                                            // [S_LABELS]
-
-    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int slice = blockIdx.x, chunk = blockIdx.y;
-    const int col = slice * SW + lane * CPL;
-    const bool col_ok = col < p.D;
-
-    for (int e = tid; e < NACC * KG * SW; e += S_THREADS) acc[e] = 0.0;
-    for (int e = tid; e < KG; e += S_THREADS) cnt[e] = 0;
-
-    const int64_t r_begin = (int64_t)chunk * p.rows_per_chunk;
-    int64_t r_end = r_begin + p.rows_per_chunk;
-    if (r_end > p.N) r_end = p.N;
-
-    for (int64_t b = r_begin; b < r_end; b += S_LABELS) {
-        __syncthreads();
-        for (int e = tid; e < S_LABELS; e += S_THREADS) {
-            int64_t r = b + e;
-            int l = (r < r_end) ? p.labels[r] : -1;
-            lab_s[e] = (l >= 0 && l < p.K) ? l : -1;
-        }
-        __syncthreads();
-        int nb = (int)((r_end - b < S_LABELS) ? (r_end - b) : S_LABELS);
-        for (int base = 0; base < nb; base += 32) {
-            int l = lab_s[base + lane];
-            int64_t row = b + base + lane;
-            int v = (l >= 0) ? l * p.copies + (int)(row % p.copies) : -1;
-            unsigned m = __ballot_sync(0xffffffffu, v >= 0 && (v % S_WARPS) == w);
-            while (m) {
-                int vv[4];
-                int64_t rr[4];
-                float q[4][CPL], f[4][CPL];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (m) {
-                        int bit = __ffs(m) - 1;
-                        m &= m - 1;
-                        vv[u] = __shfl_sync(0xffffffffu, v, bit);
-                        rr[u] = b + base + bit;
-                    } else {
-                        vv[u] = -1;
-                        rr[u] = 0;
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (vv[u] >= 0 && col_ok) {
-                        const float *src = p.Y + (size_t)rr[u] * p.D + col;
-                        load_cols<CPL>(src, q[u]);
-                        if (CENTRED) {
-                            const float *srf = p.F + (size_t)rr[u] * p.D + col;
-                            load_cols<CPL>(srf, f[u]);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (vv[u] < 0) continue;
-                    if (!CENTRED && lane == 0 && slice == 0) cnt[vv[u]]++;
-                    if (!col_ok) continue;
-                    double *a0 = acc + ((size_t)vv[u] * SW + lane * CPL);
-                    if (!CENTRED) {
-#pragma unroll
-                        for (int c = 0; c < CPL; ++c) a0[c] += (double)q[u][c];
-                    } else {
-                        int l = vv[u] / p.copies;
-                        const double *mq = p.meanQ + (size_t)l * p.D + col;
-                        const double *mf = p.meanF + (size_t)l * p.D + col;
-#pragma unroll
-                        for (int c = 0; c < CPL; ++c) {
-                            double dq = (double)q[u][c] - mq[c];
-                            double df = (double)f[u][c] - mf[c];
-                            if (NACC == 2) {
-                                a0[c] = fma(dq, dq, a0[c]);
-                                a0[(size_t)KG * SW + c] = fma(dq, df, a0[(size_t)KG * SW + c]);
-                            } else if (p.mask == 1) {
-                                a0[c] = fma(dq, dq, a0[c]);
-                            } else {
-                                a0[c] = fma(dq, df, a0[c]);
-                            }
-                        }
-                    }
-                }
-            }
-        }
-    }
-    __syncthreads();
-
-    // fold the copies and publish this CTA's partial sums
-    const size_t KD = (size_t)p.K * p.D;
-    for (int e = tid; e < NACC * p.K * SW; e += S_THREADS) {
-        int a = e / (p.K * SW);
-        int rem = e - a * (p.K * SW);
-        int k = rem / SW, c = rem - k * SW;
-        int gc = slice * SW + c;
-        if (gc >= p.D) continue;
-        double s = 0.0;
-        for (int g = 0; g < p.copies; ++g) s += acc[((size_t)a * KG + (size_t)k * p.copies + g) * SW + c];
-        int plane = (NACC == 2) ? a : ((CENTRED && p.mask == 2) ? 1 : 0);
-        p.partial[((size_t)chunk * 2 + plane) * KD + (size_t)k * p.D + gc] = s;
-    }
-    if (!CENTRED && slice == 0) {
-        for (int k = tid; k < p.K; k += S_THREADS) {
-            int s = 0;
-            for (int g = 0; g < p.copies; ++g) s += cnt[k * p.copies + g];
-            p.partial_cnt[(size_t)chunk * p.K + k] = s;
-        }
-    }
-}
-
-template <int CPL, int NACC, bool CENTRED>
-static cudaError_t launch_partial_t(const SumParams &p, const SumGeom &g, cudaStream_t s)
-{
-    auto kern = cluster_partial_kernel<CPL, NACC, CENTRED>;
-    static size_t configured[kMaxDevices] = {};  // the attribute is kept per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = -1;
-    if (dev < 0 || g.smem_bytes > configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)g.smem_bytes);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0) configured[dev] = g.smem_bytes;
-    }
-    dim3 grid((unsigned)g.nslices, (unsigned)g.nchunks);
-    kern<<<grid, S_THREADS, g.smem_bytes, s>>>(p);
-    count_launch();
-    return cudaGetLastError();
-}
-
-cudaError_t launch_cluster_partial(const float *Y, const float *F, const int32_t *labels,
-                                   int64_t N, int D, int K, const SumGeom &g,
-                                   const double *meanQ, const double *meanF, int mask,
-                                   double *partial, int32_t *partial_cnt, cudaStream_t s)
-{
-    SumParams p{Y, F, labels, meanQ, meanF, partial, partial_cnt, N, g.rows_per_chunk,
-                D, K, g.copies, mask};
-    const bool centred = (mask != 0);
-    if (!centred) {
-        switch (g.cpl) {
-        case 4: return launch_partial_t<4, 1, false>(p, g, s);
-        case 2: return launch_partial_t<2, 1, false>(p, g, s);
-        default: return launch_partial_t<1, 1, false>(p, g, s);
-        }
-    }
-    if (g.nacc == 2) {
-        switch (g.cpl) {
-        case 4: return launch_partial_t<4, 2, true>(p, g, s);
-        case 2: return launch_partial_t<2, 2, true>(p, g, s);
-        default: return launch_partial_t<1, 2, true>(p, g, s);
-        }
-    }
-    switch (g.cpl) {
-    case 4: return launch_partial_t<4, 1, true>(p, g, s);
-    case 2: return launch_partial_t<2, 1, true>(p, g, s);
-    default: return launch_partial_t<1, 1, true>(p, g, s);
-    }
-}
-
-// ======================================================================================
 // element-wise kernels
 // ======================================================================================
-
-__global__ void reduce_partials_kernel(const double *__restrict__ partial,
-                                       const int32_t *__restrict__ partial_cnt, int nchunks,
-                                       int plane, size_t KD, int K, double *__restrict__ out,
-                                       int64_t *__restrict__ counts)
-{
-    size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e < KD) {
-        double s = 0.0;
-        for (int c = 0; c < nchunks; ++c) s += partial[((size_t)c * 2 + plane) * KD + e];
-        out[e] = s;
-    }
-    if (counts && e < (size_t)K) {
-        int64_t s = 0;
-        for (int c = 0; c < nchunks; ++c) s += partial_cnt[(size_t)c * K + e];
-        counts[e] = s;
-    }
-}
-
-cudaError_t launch_reduce_partials(const double *partial, const int32_t *partial_cnt, int nchunks,
-                                   int nplanes, int plane, int D, int K, double *out,
-                                   int64_t *counts, cudaStream_t s)
-{
-    (void)nplanes;
-    size_t KD = (size_t)K * D;
-    int threads = 256;
-    unsigned blocks = (unsigned)((KD + threads - 1) / threads);
-    reduce_partials_kernel<<<blocks, threads, 0, s>>>(partial, partial_cnt, nchunks, plane, KD, K,
-                                                      out, counts);
-    count_launch();
-    return cudaGetLastError();
-}
 
 __global__ void centroids_from_sums_kernel(const double *__restrict__ sums,
                                            const int64_t *__restrict__ counts, int D, size_t KD,

@@ -1,0 +1,379 @@
+// Segmented (per-cluster) sums through a stable sort of the rows by label.
+//
+//   label_hist_kernel     per-block label histograms (1024 rows per block)
+//   label_scan_kernel     cluster sizes, cluster offsets, per-block offsets, segment table
+//   label_scatter_kernel  stable scatter of the row indices: order[] lists the rows of
+//                         cluster 0 in ascending row order, then cluster 1, ...
+//   segment_sums_kernel   one CTA per segment (<= seg_rows consecutive entries of order[], all of
+//                         one cluster): streams those rows with 128-bit loads and keeps the
+//                         column sums in fp64 registers -- no atomics, no shared accumulators,
+//                         fixed summation order -- and writes one partial row per segment
+//   segment_combine_kernel  adds a cluster's segment partials in order; optionally turns the
+//                         sums into centroids
+//
+// Three reductions use the same machinery: column sums of one matrix (a Lloyd round), of
+// two matrices (the final pass: sums of Yq and Yfp), and the centred second moments
+// sum (q - muQ)^2, sum (q - muQ)(f - muF) with the cluster means held in registers.
+#include "cat_internal.cuh"
+
+namespace cat {
+
+namespace {
+
+constexpr int SORT_BLOCK = 1024;     // rows per histogram / scatter block
+constexpr int SEG_THREADS = 256;
+
+__global__ void __launch_bounds__(SORT_BLOCK) label_hist_kernel(const int32_t *__restrict__ labels, int64_t N,
+                                                                 int K, uint32_t *__restrict__ blk_hist)
+{
+    extern __shared__ uint32_t hist[];   // [K]
+    for (int k = threadIdx.x; k < K; k += SORT_BLOCK) hist[k] = 0;
+    __syncthreads();
+    const int64_t row = (int64_t)blockIdx.x * SORT_BLOCK + threadIdx.x;
+    if (row < N) {
+        const int l = labels[row];
+        if (l >= 0 && l < K) atomicAdd(&hist[l], 1u);
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < K; k += SORT_BLOCK) blk_hist[(size_t)blockIdx.x * K + k] = hist[k];
+}
+
+// One CTA.  Thread k walks the blocks of cluster k: blk_hist[b][k] becomes the number of rows
+// of cluster k in blocks before b.  Then cluster_start (exclusive scan of the sizes) and
+// seg_start (exclusive scan of ceil(size / seg_rows)), each with K + 1 entries.
+__global__ void __launch_bounds__(512) label_scan_kernel(uint32_t *__restrict__ blk_hist, int nblk, int K,
+                                                         int seg_rows, int64_t *__restrict__ counts,
+                                                         int32_t *__restrict__ cluster_start,
+                                                         int32_t *__restrict__ seg_start)
+{
+    __shared__ uint32_t size_s[CAT_MAX_K];
+    const int k = threadIdx.x;
+    uint32_t run = 0;
+    if (k < K) {
+        for (int b = 0; b < nblk; ++b) {
+            const size_t o = (size_t)b * K + k;
+            const uint32_t v = blk_hist[o];
+            blk_hist[o] = run;
+            run += v;
+        }
+        counts[k] = (int64_t)run;
+        size_s[k] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t a = 0, sgs = 0;
+        for (int q = 0; q < K; ++q) {
+            cluster_start[q] = (int32_t)a;
+            seg_start[q] = (int32_t)sgs;
+            a += size_s[q];
+            sgs += (size_s[q] + (uint32_t)seg_rows - 1) / (uint32_t)seg_rows;
+        }
+        cluster_start[K] = (int32_t)a;
+        seg_start[K] = (int32_t)sgs;
+    }
+}
+
+// Stable scatter.  Within a block, a row's rank among the rows of its cluster is
+// (rows of that cluster in earlier warps) + (rows of that cluster in earlier lanes).
+__global__ void __launch_bounds__(SORT_BLOCK) label_scatter_kernel(const int32_t *__restrict__ labels, int64_t N,
+                                                                    int K, const uint32_t *__restrict__ blk_hist,
+                                                                    const int32_t *__restrict__ cluster_start,
+                                                                    int32_t *__restrict__ order)
+{
+    extern __shared__ uint16_t warp_hist[];   // [32][K]
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    for (int e = tid; e < 32 * K; e += SORT_BLOCK) warp_hist[e] = 0;
+    __syncthreads();
+    const int64_t row = (int64_t)blockIdx.x * SORT_BLOCK + tid;
+    int l = -1;
+    if (row < N) {
+        l = labels[row];
+        if (l < 0 || l >= K) l = -1;
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, l);
+    const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+    if (l >= 0 && rank_in_warp == 0) warp_hist[w * K + l] = (uint16_t)__popc(peers);
+    __syncthreads();
+    for (int k = tid; k < K; k += SORT_BLOCK) {
+        uint16_t run = 0;
+        for (int q = 0; q < 32; ++q) {
+            const uint16_t v = warp_hist[q * K + k];
+            warp_hist[q * K + k] = run;
+            run = (uint16_t)(run + v);
+        }
+    }
+    __syncthreads();
+    if (l >= 0) {
+        const uint32_t pos = (uint32_t)cluster_start[l] + blk_hist[(size_t)blockIdx.x * K + l] +
+                             warp_hist[w * K + l] + (uint32_t)rank_in_warp;
+        order[pos] = (int32_t)row;
+    }
+}
+
+struct SegParams {
+    const float *Yq;
+    const float *Yf;            // second matrix (modes 1, 2)
+    const int32_t *order;
+    const int32_t *cluster_start;
+    const int32_t *seg_start;
+    const double *meanQ;        // mode 2
+    const double *meanF;
+    double *part;               // [maxsegs][2][D]
+    int D;
+    int K;
+    int seg_rows;
+    int tpr;                    // threads per row (power of two <= 256)
+};
+
+__device__ __forceinline__ void add4(double (&a)[4], const float4 v)
+{
+    a[0] += (double)v.x;
+    a[1] += (double)v.y;
+    a[2] += (double)v.z;
+    a[3] += (double)v.w;
+}
+
+// MODE 0: sums of Yq -> plane 0.  MODE 1: sums of Yq, Yf -> planes 0, 1.
+// MODE 2: centred moments -> plane 0 = sum (q-muQ)^2, plane 1 = sum (q-muQ)(f-muF).
+// VEC: 4 = 128-bit loads (D % 4 == 0), 1 = scalar loads.
+template <int MODE, int VEC>
+__global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
+{
+    __shared__ int32_t rows_s[128];
+    __shared__ double red_s[SEG_THREADS * VEC];
+    const int seg = blockIdx.x;
+    const int nseg_total = p.seg_start[p.K];
+    if (seg >= nseg_total) return;
+    // cluster of this segment: last k with seg_start[k] <= seg
+    int lo = 0, hi = p.K;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (p.seg_start[mid] <= seg) lo = mid; else hi = mid;
+    }
+    const int k = lo;
+    const int first = p.cluster_start[k] + (seg - p.seg_start[k]) * p.seg_rows;
+    int nrows = p.cluster_start[k + 1] - first;
+    if (nrows > p.seg_rows) nrows = p.seg_rows;
+
+    const int tid = threadIdx.x;
+    const int tpr = p.tpr;
+    const int c = tid & (tpr - 1);      // column unit within the block of columns
+    const int g = tid / tpr;            // row group
+    const int G = SEG_THREADS / tpr;
+    const int units = (p.D + VEC - 1) / VEC;          // column units per row
+    const int col0 = blockIdx.y * SEG_THREADS;        // first unit of this column block
+    const int unit = col0 + c;
+    const bool active = (c < SEG_THREADS) && (unit < units);
+    const int col = unit * VEC;
+
+    double a0[4] = {0, 0, 0, 0}, a1[4] = {0, 0, 0, 0};
+    double mq[4] = {0, 0, 0, 0}, mf[4] = {0, 0, 0, 0};
+    if (MODE == 2 && active) {
+#pragma unroll
+        for (int q = 0; q < VEC; ++q) {
+            mq[q] = p.meanQ[(size_t)k * p.D + col + q];
+            mf[q] = p.meanF[(size_t)k * p.D + col + q];
+        }
+    }
+
+    for (int base = 0; base < nrows; base += 128) {
+        const int nb = (nrows - base < 128) ? (nrows - base) : 128;
+        __syncthreads();
+        if (tid < nb) rows_s[tid] = p.order[first + base + tid];
+        __syncthreads();
+        if (!active) continue;
+        int r = g;
+        // four rows in flight per thread
+        for (; r + 3 * G < nb; r += 4 * G) {
+            float4 q4[4], f4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const size_t o = (size_t)rows_s[r + u * G] * p.D + col;
+                if (VEC == 4) {
+                    q4[u] = __ldg(reinterpret_cast<const float4 *>(p.Yq + o));
+                    if (MODE != 0) f4[u] = __ldg(reinterpret_cast<const float4 *>(p.Yf + o));
+                } else {
+                    q4[u] = make_float4(__ldg(p.Yq + o), 0.f, 0.f, 0.f);
+                    if (MODE != 0) f4[u] = make_float4(__ldg(p.Yf + o), 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (MODE == 0) {
+                    add4(a0, q4[u]);
+                } else if (MODE == 1) {
+                    add4(a0, q4[u]);
+                    add4(a1, f4[u]);
+                } else {
+                    const float qv[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
+                    const float fv[4] = {f4[u].x, f4[u].y, f4[u].z, f4[u].w};
+#pragma unroll
+                    for (int q = 0; q < VEC; ++q) {
+                        const double dq = (double)qv[q] - mq[q];
+                        const double df = (double)fv[q] - mf[q];
+                        a0[q] = fma(dq, dq, a0[q]);
+                        a1[q] = fma(dq, df, a1[q]);
+                    }
+                }
+            }
+        }
+        for (; r < nb; r += G) {
+            const size_t o = (size_t)rows_s[r] * p.D + col;
+            float4 q4, f4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (VEC == 4) {
+                q4 = __ldg(reinterpret_cast<const float4 *>(p.Yq + o));
+                if (MODE != 0) f4 = __ldg(reinterpret_cast<const float4 *>(p.Yf + o));
+            } else {
+                q4 = make_float4(__ldg(p.Yq + o), 0.f, 0.f, 0.f);
+                if (MODE != 0) f4 = make_float4(__ldg(p.Yf + o), 0.f, 0.f, 0.f);
+            }
+            if (MODE == 0) {
+                add4(a0, q4);
+            } else if (MODE == 1) {
+                add4(a0, q4);
+                add4(a1, f4);
+            } else {
+                const float qv[4] = {q4.x, q4.y, q4.z, q4.w};
+                const float fv[4] = {f4.x, f4.y, f4.z, f4.w};
+#pragma unroll
+                for (int q = 0; q < VEC; ++q) {
+                    const double dq = (double)qv[q] - mq[q];
+                    const double df = (double)fv[q] - mf[q];
+                    a0[q] = fma(dq, dq, a0[q]);
+                    a1[q] = fma(dq, df, a1[q]);
+                }
+            }
+        }
+    }
+
+    // add the row groups in a fixed order and publish the segment's partial row
+    constexpr int NPLANES = (MODE == 0) ? 1 : 2;
+#pragma unroll
+    for (int pl = 0; pl < NPLANES; ++pl) {
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < VEC; ++q) red_s[tid * VEC + q] = (pl == 0) ? a0[q] : a1[q];
+        __syncthreads();
+        if (g == 0 && active) {
+            double *dst = p.part + ((size_t)seg * 2 + pl) * p.D + col;
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) {
+                double s = 0.0;
+                for (int gg = 0; gg < G; ++gg) s += red_s[(gg * tpr + c) * VEC + q];
+                dst[q] = s;
+            }
+        }
+    }
+}
+
+// out0/out1[k*D+j] = sum over the segments of cluster k of plane 0/1 (out1 may be NULL);
+// with C != NULL also C[k*D+j] = float(out0 / n_k) where n_k > 0.
+__global__ void segment_combine_kernel(const double *__restrict__ part, const int32_t *__restrict__ seg_start,
+                                       const int64_t *__restrict__ counts, int D, size_t KD,
+                                       double *__restrict__ out0, double *__restrict__ out1,
+                                       float *__restrict__ C)
+{
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= KD) return;
+    const int k = (int)(e / D);
+    const int j = (int)(e - (size_t)k * D);
+    const int s0 = seg_start[k], s1 = seg_start[k + 1];
+    double a = 0.0, b = 0.0;
+    for (int sgm = s0; sgm < s1; ++sgm) {
+        a += part[((size_t)sgm * 2) * D + j];
+        if (out1) b += part[((size_t)sgm * 2 + 1) * D + j];
+    }
+    out0[e] = a;
+    if (out1) out1[e] = b;
+    if (C) {
+        const int64_t n = counts[k];
+        if (n > 0) C[e] = (float)(a / (double)n);
+    }
+}
+
+int tpr_for(int units)
+{
+    int t = 1;
+    while (t < units && t < SEG_THREADS) t <<= 1;
+    return t;
+}
+
+}  // namespace
+
+SegGeom seg_geometry(int64_t N, int D, int K)
+{
+    SegGeom g{};
+    g.nblk = (int)((N + SORT_BLOCK - 1) / SORT_BLOCK);
+    int64_t sr = (N + 2047) / 2048;
+    if (sr < 128) sr = 128;
+    sr = (sr + 127) / 128 * 128;
+    g.seg_rows = (int)sr;
+    g.max_segs = (int)((N + sr - 1) / sr) + K;
+    (void)D;
+    return g;
+}
+
+cudaError_t launch_label_sort(const int32_t *labels, int64_t N, int K, const SegGeom &g, uint32_t *blk_hist,
+                              int64_t *counts, int32_t *cluster_start, int32_t *seg_start, int32_t *order,
+                              cudaStream_t s)
+{
+    label_hist_kernel<<<g.nblk, SORT_BLOCK, (size_t)K * sizeof(uint32_t), s>>>(labels, N, K, blk_hist);
+    label_scan_kernel<<<1, 512, 0, s>>>(blk_hist, g.nblk, K, g.seg_rows, counts, cluster_start, seg_start);
+    label_scatter_kernel<<<g.nblk, SORT_BLOCK, (size_t)32 * K * sizeof(uint16_t), s>>>(labels, N, K, blk_hist,
+                                                                                       cluster_start, order);
+    count_launch(3);
+    return cudaGetLastError();
+}
+
+template <int MODE>
+static cudaError_t launch_segment_sums_mode(const SegParams &p, const SegGeom &g, cudaStream_t s)
+{
+    const bool vec = (p.D % 4 == 0);
+    const int units = vec ? p.D / 4 : p.D;
+    dim3 grid((unsigned)g.max_segs, (unsigned)((units + SEG_THREADS - 1) / SEG_THREADS));
+    if (vec)
+        segment_sums_kernel<MODE, 4><<<grid, SEG_THREADS, 0, s>>>(p);
+    else
+        segment_sums_kernel<MODE, 1><<<grid, SEG_THREADS, 0, s>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, const int32_t *order,
+                                const int32_t *cluster_start, const int32_t *seg_start, const double *meanQ,
+                                const double *meanF, int D, int K, const SegGeom &g, double *part,
+                                cudaStream_t s)
+{
+    SegParams p{};
+    p.Yq = Yq;
+    p.Yf = Yf;
+    p.order = order;
+    p.cluster_start = cluster_start;
+    p.seg_start = seg_start;
+    p.meanQ = meanQ;
+    p.meanF = meanF;
+    p.part = part;
+    p.D = D;
+    p.K = K;
+    p.seg_rows = g.seg_rows;
+    const int units = (D % 4 == 0) ? D / 4 : D;
+    p.tpr = tpr_for(units);
+    switch (mode) {
+    case 0: return launch_segment_sums_mode<0>(p, g, s);
+    case 1: return launch_segment_sums_mode<1>(p, g, s);
+    default: return launch_segment_sums_mode<2>(p, g, s);
+    }
+}
+
+cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
+                                   int K, double *out0, double *out1, float *C, cudaStream_t s)
+{
+    const size_t KD = (size_t)K * D;
+    const int threads = 256;
+    const unsigned blocks = (unsigned)((KD + threads - 1) / threads);
+    segment_combine_kernel<<<blocks, threads, 0, s>>>(part, seg_start, counts, D, KD, out0, out1, C);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace cat

@@ -1,21 +1,31 @@
 // Tensor-core path of the nearest-centroid assignment (sm_100a: tcgen05 + TMEM + TMA).
 //
-// The N x K x D distance contraction y_i . c_k runs as a TF32 UMMA: a persistent CTA
-// walks 128-row tiles; TMA streams 128 x 32 fp32 slabs of the rows and K x 32 slabs of
-// the centroids into 128-byte-swizzled shared memory, one thread issues
+// The N x K x D distance contraction y_i . c_k runs as a TF32 UMMA.  A persistent CTA
+// walks 128-row tiles; TMA streams 128 x 32 fp32 slabs of the rows and slabs of the
+// centroids into 128-byte-swizzled shared memory, one thread issues
 // tcgen05.mma.kind::tf32 into a TMEM accumulator (128 lanes x K columns, two buffers),
-// and the epilogue warps read the scores back with tcgen05.ld, take best / second /
-// argmin per row and run the same certainty test as the fp32 path, with the TF32 error
-// bound
-//     e <= (2^-8 + (2D+2) 2^-22) ||y|| cmax + 4 u cmax^2
-// (operands cut to 11 significant bits: <= 2^-10 each; fp32 accumulation inside the
-// tensor core taken as <= 2^-22 per term).  Rows it cannot decide go to the same exact
-// fp64 pass, so labels stay exact.  For inference the epilogue then streams each decided
-// row once more (it is still in L2) and writes gamma_l * y + beta_l.
+// and the score warps read the scores back with tcgen05.ld and keep the four smallest per
+// row.  With more than one tile of rows the CTAs work in pairs (cta_group::2, M = 256):
+// each CTA of a pair stages its own 128 rows and HALF the centroids, which halves the
+// centroid bytes that leave L2 per row.
 //
-// Every wait on an mbarrier is bounded (about 2 s): on a timeout the CTA records
-// CAT_ERR_DEVICE_TIMEOUT in the control block, all roles leave their loops, outstanding
-// copies and MMAs are drained with bounded waits, TMEM is freed and the kernel returns.
+// A score travels as a "key": its fp32 bits with the low 8 bits replaced by the centroid
+// index, so that the four smallest come out of a branch-free min/max insertion network.
+// The certainty test is the one of the fp32 path with the error bound
+//     e <= (2^-8 + (2D+2) 2^-22) ||y|| cmax + 4 u cmax^2 + 2^-15 (cmax^2 + 2 ||y|| cmax)
+// (operands cut to 11 significant bits: <= 2^-10 each; fp32 accumulation inside the
+// tensor core taken as <= 2^-22 per term; the last term is the index packed into the
+// key).  Rows it cannot decide go to the same exact fp64 pass, so labels stay exact.
+//
+// For inference, streaming warps then read every row of the tile once more and write
+// gamma_l * y + beta_l for the fast label l; an undecided row is queued and the exact pass
+// rewrites its output.  The TMA producer may run at most one tile ahead of the streaming
+// warps, which bounds the bytes between a row's first read and its second.
+//
+// Every wait on an mbarrier or a progress counter is bounded (about 2 s): on a timeout the
+// CTA records CAT_ERR_DEVICE_TIMEOUT in the control block, all roles leave their loops,
+// outstanding copies and MMAs are drained with bounded waits, TMEM is freed and the kernel
+// returns.
 #include "cat_internal.cuh"
 
 #include <cuda.h>
@@ -25,13 +35,35 @@ namespace cat {
 
 namespace {
 
-constexpr int TC_BM = 128;                   // rows per tile (UMMA M)
+constexpr int TC_BM = 128;                   // rows per CTA tile (UMMA M per CTA)
 constexpr int TC_BK = 32;                    // fp32 per slab = 128 B = one swizzle row
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 4;  // 16 KB
-constexpr int TC_STAGES = 4;
-constexpr int TC_SCORE_WARPS = 4;
-constexpr int TC_STREAM_WARPS = 12;          // AFFINE only; includes the 4 score warps
+constexpr int TC_MAX_STAGES = 8;
 constexpr uint64_t TC_TIMEOUT_NS = 2000000000ull;
+
+// Warp roles.  Warp 0: TMA producer, warp 1: MMA issuer (2, 3 idle), warps 4-7: score warps
+// (TMEM lane quarter = warp & 3); with the affine epilogue also warps 8-19: streaming warps.
+constexpr int TC_FIRST_SCORE_WARP = 4;
+constexpr int TC_SCORE_WARPS = 4;
+constexpr int TC_FIRST_STREAM_WARP = 8;
+constexpr int TC_STREAM_WARPS = 12;
+constexpr int TC_THREADS_LABELS = 32 * TC_FIRST_STREAM_WARP;                       // 256
+constexpr int TC_THREADS_AFFINE = 32 * (TC_FIRST_STREAM_WARP + TC_STREAM_WARPS);   // 640
+// Register split of the affine kernel (per thread, by warpgroup of 128 threads): the kernel
+// is launched with TC_REGS_LAUNCH registers per thread; the producer/MMA warpgroup and the
+// score warpgroup give registers back, the three streaming warpgroups take them.  The shares
+// add up to no more than the launch total (checked again on the host before every launch).
+constexpr int TC_REGS_LAUNCH = 96;
+constexpr int TC_REGS_CONTROL = 24;
+constexpr int TC_REGS_SCORE = 72;
+constexpr int TC_REGS_STREAM = 128;
+static_assert(128 * (TC_REGS_CONTROL + TC_REGS_SCORE + 3 * TC_REGS_STREAM) <= TC_REGS_LAUNCH * TC_THREADS_AFFINE,
+              "register split exceeds what the block is launched with");
+// The streaming warps read through L1, and the number of loads an SM keeps in flight shrinks
+// with L1: a shared-memory carve-out of 200 KB and more costs a third of the streaming rate
+// (measured), about 100 KB costs nothing.  The tile period of the affine kernel is long
+// enough for a shallow TMA ring, so that kernel takes the smaller carve-out.
+constexpr int TC_AFFINE_MAX_STAGES = 3;
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -68,7 +100,9 @@ __device__ __forceinline__ uint64_t global_timer()
 }
 
 // Bounded wait.  Returns false after a timeout or once another role has given up.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, Control *ctl)
+// (Inlined on purpose: a called function inside the re-divided register budgets of the
+// affine kernel sends ptxas into a very long compile.)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, Control *ctl)
 {
     uint64_t t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -94,6 +128,26 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     return __all_sync(0xffffffffu, ok);
 }
 
+// Bounded wait until *counter >= need.  Returns false after a timeout or an abort.
+__device__ __forceinline__ bool wait_progress(volatile int *counter, int need, volatile int *abort_flag, Control *ctl)
+{
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (*counter >= need) return true;
+        if (*abort_flag) return false;
+        if ((it & 63u) == 63u) {
+            uint64_t now = global_timer();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > TC_TIMEOUT_NS) {
+                *abort_flag = 1;
+                atomicExch(&ctl->device_status, (int)CAT_ERR_DEVICE_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
 {
     asm volatile(
@@ -117,9 +171,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
 __device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
@@ -130,20 +181,103 @@ __device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64
         : "memory");
 }
 
-// 16 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
+// ---- cluster / cta_group::2 forms (every tcgen05 instruction of a kernel uses one cta_group)
+__device__ __forceinline__ uint32_t cluster_ctarank()
 {
-    uint32_t r[16];
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory location in the CTA of the given rank
+__device__ __forceinline__ uint32_t mapa_cluster(uint32_t cta_addr, uint32_t rank)
+{
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(cta_addr), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load whose completion is reported to a barrier that may live in the peer CTA of the pair
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t cluster_bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(cluster_bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
+        ::"r"(bar)
+        : "memory");
+}
+// arrives on this CTA's barrier only
+__device__ __forceinline__ void tc_commit_pair_local(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mma_tf32_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+template <int R>
+__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(R)); }
+template <int R>
+__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(R)); }
+
+// 16 consecutive fp32 columns of this thread's TMEM lane.  The load is asynchronous: the
+// registers hold the data only after tmem_ld_wait16 on the same array, which also keeps
+// the compiler from reading them any earlier.
+#define CAT_OUT(x) "=r"(x)
+#define CAT_INOUT(x) "+r"(x)
+#define CAT_R16(r, o) o(r[0]), o(r[1]), o(r[2]), o(r[3]), o(r[4]), o(r[5]), o(r[6]), o(r[7]), o(r[8]), o(r[9]), \
+    o(r[10]), o(r[11]), o(r[12]), o(r[13]), o(r[14]), o(r[15])
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16])
+{
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : CAT_R16(r, CAT_OUT)
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : CAT_R16(r, CAT_INOUT)::"memory");
 }
 
 // K-major, 128-byte-swizzled operand tile whose rows are 128 B apart: 8-row groups every
@@ -159,11 +293,25 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr)
     return d;
 }
 
-// D = F32, A = B = TF32, both K-major, M = 128, N = n.
-__host__ __device__ constexpr uint32_t make_idesc_tf32(int n)
+// D = F32, A = B = TF32, both K-major, M = m (128, or 256 over a CTA pair), N = n.
+__host__ __device__ constexpr uint32_t make_idesc_tf32(int m, int n)
 {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
+
+// Optional timeline of the first two CTAs (compiled in only with -DCAT_TC_TRACE): globaltimer
+// stamps per role and tile, read back with cat_tc_trace_read.
+#ifdef CAT_TC_TRACE
+constexpr int TC_TRACE_TILES = 16;
+constexpr int TC_TRACE_EVENTS = 8;
+__device__ unsigned long long g_tc_trace[2][TC_TRACE_TILES][TC_TRACE_EVENTS];
+#define TC_TRACE(ti, ev)                                                                               \
+    do {                                                                                               \
+        if (blockIdx.x < 2 && (ti) < TC_TRACE_TILES) g_tc_trace[blockIdx.x][ti][ev] = global_timer();  \
+    } while (0)
+#else
+#define TC_TRACE(ti, ev) do { } while (0)
+#endif
 
 struct TcParams {
     const float *Y;
@@ -180,13 +328,14 @@ struct TcParams {
     int64_t N;
     int D;
     int K;
-    int npad;       // K rounded up to 16
-    int tmem_cols;  // power of two >= 2 * npad, >= 32
+    int npad;       // K rounded up to 32 (the score warps read TMEM 32 columns per step)
+    int tmem_cols;  // power of two >= 2 * npad
+    int stages;     // shared-memory pipeline stages (<= TC_MAX_STAGES)
 };
 
 struct TcShared {
-    uint64_t full[TC_STAGES];
-    uint64_t empty[TC_STAGES];
+    uint64_t full[TC_MAX_STAGES];
+    uint64_t empty[TC_MAX_STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t lab_full[2];
@@ -194,23 +343,51 @@ struct TcShared {
     uint64_t drain;
     uint32_t tmem_base;
     int abort_flag;
-    float red[16];
+    int rows_streamed;            // row slots the streaming warps have finished, all tiles
+    float red[32];
     float cn[256];
-    float4 top_score[2][TC_BM];   // four smallest scores of each row, ascending
-    int4 top_idx[2][TC_BM];       // their centroid indices
+    float4 top_key[2][TC_BM];     // four smallest keys of each row, ascending
 };
+
+constexpr float TC_KEY_INIT = 3.0e38f;   // larger than any finite score's key
+
+// key = score with the centroid index in the low 8 mantissa bits
+__device__ __forceinline__ float make_key(float sc, int n)
+{
+    return __uint_as_float((__float_as_uint(sc) & 0xFFFFFF00u) | (uint32_t)n);
+}
+__device__ __forceinline__ int key_index(float key) { return (int)(__float_as_uint(key) & 0xFFu); }
+
+// fast label of a row: index of its smallest key (0 if no centroid ever won, e.g. all NaN)
+__device__ __forceinline__ int key_label(float key, int K)
+{
+    const int l = key_index(key);
+    return l < K ? l : 0;
+}
+
+// keeps (b1 <= b2 <= b3 <= b4) the four smallest keys seen
+__device__ __forceinline__ void key_insert(float key, float &b1, float &b2, float &b3, float &b4)
+{
+    float t;
+    t = fminf(b1, key); key = fmaxf(b1, key); b1 = t;
+    t = fminf(b2, key); key = fmaxf(b2, key); b2 = t;
+    t = fminf(b3, key); key = fmaxf(b3, key); b3 = t;
+    b4 = fminf(b4, key);
+}
 
 __device__ __forceinline__ float tc_error_bound(int D, float ysq, float cmax2)
 {
     const float u = 5.9604645e-8f;   // 2^-24
     const float a = 3.90625e-3f + (2.f * (float)D + 2.f) * 2.3841858e-7f;  // 2^-8 + (2D+2) 2^-22
-    return 1.0625f * (a * sqrtf(ysq) * sqrtf(cmax2) + 4.f * u * cmax2);
+    const float pk = 3.0517578e-5f;                                         // 2^-15: index packed into the key
+    const float yc = sqrtf(ysq) * sqrtf(cmax2);
+    return 1.0625f * ((a + 2.f * pk) * yc + (4.f * u + pk) * cmax2);
 }
 
-// Decision for one row from its four smallest scores.  Returns true when the fast argmin is
-// certainly exact.  Otherwise the row is queued: with the centroids whose score lies within
+// Decision for one row from its four smallest keys.  Returns true when the fast argmin is
+// certainly exact.  Otherwise the row is queued: with the centroids whose key lies within
 // 2e of the best when those are known to be among the four, else for a scan of all K.
-__device__ __forceinline__ bool tc_decide(const TcParams &p, int64_t row, float4 sc, int4 id, float e)
+__device__ __forceinline__ bool tc_decide(const TcParams &p, int64_t row, float4 sc, float e)
 {
     const float lim = 2.f * e;
     if (p.K == 1 || (sc.y - sc.x) > lim) return true;
@@ -219,9 +396,9 @@ __device__ __forceinline__ bool tc_decide(const TcParams &p, int64_t row, float4
         int slot = atomicAdd(&p.ctl->refine_count, 1);
         p.refine_rows[slot] = (int32_t)row;
     } else {
-        uint64_t c = (uint64_t)(uint16_t)id.x | ((uint64_t)(uint16_t)id.y << 16);
-        c |= (uint64_t)(((sc.z - sc.x) > lim || p.K < 3) ? 0xFFFFu : (uint16_t)id.z) << 32;
-        c |= (uint64_t)(((sc.w - sc.x) > lim || p.K < 4) ? 0xFFFFu : (uint16_t)id.w) << 48;
+        uint64_t c = (uint64_t)(uint16_t)key_index(sc.x) | ((uint64_t)(uint16_t)key_index(sc.y) << 16);
+        c |= (uint64_t)(((sc.z - sc.x) > lim || p.K < 3) ? 0xFFFFu : (uint16_t)key_index(sc.z)) << 32;
+        c |= (uint64_t)(((sc.w - sc.x) > lim || p.K < 4) ? 0xFFFFu : (uint16_t)key_index(sc.w)) << 48;
         int slot = atomicAdd(&p.ctl->cand_count, 1);
         p.cand_rows[slot] = (int32_t)row;
         p.cand_list[slot] = c;
@@ -229,45 +406,106 @@ __device__ __forceinline__ bool tc_decide(const TcParams &p, int64_t row, float4
     return false;
 }
 
-template <bool AFFINE>
-__global__ void __launch_bounds__(AFFINE ? 32 * (2 + TC_STREAM_WARPS) : 32 * (2 + TC_SCORE_WARPS), 1)
+// One warp streams one row (1024 columns per step, all loads of a step in flight together):
+// out = gamma_l * y + beta_l for the fast label l, written whether or not the label is
+// certain (an undecided row is queued and the exact pass rewrites it); the row norm needed
+// by the certainty test is accumulated on the way.
+__device__ __forceinline__ void stream_row(const TcParams &p, int64_t row, float4 keys, float cmax2, int lane)
+{
+    const int D4 = p.D >> 2;
+    const int l = key_label(keys.x, p.K);
+    const float4 *y4 = reinterpret_cast<const float4 *>(p.Y) + (size_t)row * D4 + lane;
+    const float4 *g4 = reinterpret_cast<const float4 *>(p.gamma) + (size_t)l * D4 + lane;
+    const float4 *b4 = reinterpret_cast<const float4 *>(p.beta) + (size_t)l * D4 + lane;
+    float4 *o4 = reinterpret_cast<float4 *>(p.out) + (size_t)row * D4 + lane;
+    float ysq = 0.f;
+#pragma unroll 1
+    for (int h = 0; h < D4; h += 256) {
+        float4 y[8], g[8], bb[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int c = h + 32 * q;
+            if (c + lane < D4) {
+                y[q] = __ldcs(y4 + c);
+                g[q] = __ldg(g4 + c);
+                bb[q] = __ldg(b4 + c);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int c = h + 32 * q;
+            if (c + lane < D4) {
+                float4 v;
+                v.x = fmaf(g[q].x, y[q].x, bb[q].x);
+                v.y = fmaf(g[q].y, y[q].y, bb[q].y);
+                v.z = fmaf(g[q].z, y[q].z, bb[q].z);
+                v.w = fmaf(g[q].w, y[q].w, bb[q].w);
+                __stcs(o4 + c, v);
+                ysq = fmaf(y[q].x, y[q].x, ysq);
+                ysq = fmaf(y[q].y, y[q].y, ysq);
+                ysq = fmaf(y[q].z, y[q].z, ysq);
+                ysq = fmaf(y[q].w, y[q].w, ysq);
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
+    if (lane == 0) {
+        // the row norm enters the bound slightly over-estimated
+        const float e = tc_error_bound(p.D, ysq * 1.0001f, cmax2);
+        p.labels[row] = l;
+        tc_decide(p, row, keys, e);
+    }
+}
+
+// PAIR: the two CTAs of a cluster work as one cta_group::2 unit on 256 rows.  Each CTA
+// loads the slabs of its own 128 rows and of HALF the centroids; the MMA (M = 256, issued
+// by the CTA of rank 0) reads both halves, and each CTA finds the scores of its own rows in
+// its own TMEM.
+template <bool AFFINE, bool PAIR>
+__global__ void __launch_bounds__(AFFINE ? TC_THREADS_AFFINE : TC_THREADS_LABELS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p)
 {
-    constexpr int NEPI = AFFINE ? TC_STREAM_WARPS : TC_SCORE_WARPS;
     extern __shared__ unsigned char smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;
     unsigned char *tiles = smem_raw + (tiles_base - raw);
-    const int b_bytes = p.npad * 128;
-    const int stage_bytes = TC_A_BYTES + b_bytes;
-    TcShared &sh = *reinterpret_cast<TcShared *>(tiles + (size_t)TC_STAGES * stage_bytes);
+    const int nb_rows = PAIR ? (p.npad >> 1) : p.npad;   // centroid rows this CTA stages per slab
+    const int stage_bytes = TC_A_BYTES + nb_rows * 128;
+    const int nstages = p.stages;
+    TcShared &sh = *reinterpret_cast<TcShared *>(tiles + (size_t)nstages * stage_bytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // 0 = the CTA that issues the MMAs
     volatile int *abort_flag = &sh.abort_flag;
-    const int64_t num_tiles = (p.N + TC_BM - 1) / TC_BM;
+    // work units: 128-row tiles, or 256-row pair tiles shared by the two CTAs of a cluster
+    const int64_t num_units = PAIR ? (p.N + 2 * TC_BM - 1) / (2 * TC_BM) : (p.N + TC_BM - 1) / TC_BM;
+    const int64_t unit_first = PAIR ? (int64_t)(blockIdx.x >> 1) : (int64_t)blockIdx.x;
+    const int64_t unit_step = PAIR ? (int64_t)(gridDim.x >> 1) : (int64_t)gridDim.x;
     const int nslabs = (p.D + TC_BK - 1) / TC_BK;
 
     if (tid == 0) {
-        for (int s = 0; s < TC_STAGES; ++s) {
-            mbar_init(smem_u32(&sh.full[s]), 1);
+        for (int s = 0; s < nstages; ++s) {
+            mbar_init(smem_u32(&sh.full[s]), PAIR ? 2 : 1);    // one expect_tx arrival per CTA
             mbar_init(smem_u32(&sh.empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sh.tmem_full[b]), 1);
-            mbar_init(smem_u32(&sh.tmem_empty[b]), TC_SCORE_WARPS);
+            mbar_init(smem_u32(&sh.tmem_empty[b]), (PAIR ? 2 : 1) * TC_SCORE_WARPS);
             mbar_init(smem_u32(&sh.lab_full[b]), TC_SCORE_WARPS);
-            mbar_init(smem_u32(&sh.lab_empty[b]), NEPI);
+            mbar_init(smem_u32(&sh.lab_empty[b]), TC_STREAM_WARPS);
         }
         mbar_init(smem_u32(&sh.drain), 1);
         sh.abort_flag = 0;
+        sh.rows_streamed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // centroid norms (+inf beyond K) and their maximum
+    // centroid norms (a huge finite value beyond K) and their maximum
     {
         float m = 0.f;
         for (int k = tid; k < 256; k += blockDim.x) {
-            float v = (k < p.K) ? p.cnorm[k] : CUDART_INF_F;
+            float v = (k < p.K) ? p.cnorm[k] : TC_KEY_INIT;
             sh.cn[k] = v;
             if (k < p.K) m = fmaxf(m, v);
         }
@@ -276,223 +514,192 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         if (lane == 0) sh.red[warp] = m;
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&sh.tmem_base), (uint32_t)p.tmem_cols);
-        tmem_relinquish();
+        if (PAIR) {
+            tmem_alloc_pair(smem_u32(&sh.tmem_base), (uint32_t)p.tmem_cols);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(&sh.tmem_base), (uint32_t)p.tmem_cols);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync();   // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     float cmax2 = 0.f;
     for (int w2 = 0; w2 < (int)(blockDim.x >> 5); ++w2) cmax2 = fmaxf(cmax2, sh.red[w2]);
     const uint32_t tmem_base = sh.tmem_base;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                for (int sl = 0; sl < nslabs; ++sl, ++it) {
-                    const int s = it % TC_STAGES;
-                    const uint32_t ph = (it / TC_STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
-                    const uint32_t full = smem_u32(&sh.full[s]);
-                    mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
-                    const uint32_t a_dst = tiles_base + (uint32_t)(s * stage_bytes);
-                    tma_load_2d(a_dst, &mapA, full, sl * TC_BK, (int)(tile * TC_BM));
-                    tma_load_2d(a_dst + TC_A_BYTES, &mapB, full, sl * TC_BK, 0);
+    // With the affine epilogue each warpgroup first trades registers: the control and score
+    // warpgroups give some back, the streaming warpgroups take them.
+    if (warp < TC_FIRST_SCORE_WARP) {
+        if (AFFINE) setmaxnreg_dec<TC_REGS_CONTROL>();
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer
+            if (lane == 0) {
+                uint32_t it = 0, ti = 0;
+                bool ok = true;
+                for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
+                    const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
+                    if (AFFINE && ti > 1) {
+                        // at most one tile ahead of the streaming warps: tile ti - 2 is streamed out
+                        if (!wait_progress(&sh.rows_streamed, (int)(ti - 1) * TC_BM, abort_flag, p.ctl)) { ok = false; break; }
+                    }
+                    for (int sl = 0; sl < nslabs; ++sl, ++it) {
+                        const int s = it % nstages;
+                        const uint32_t ph = (it / nstages) & 1u;
+                        if (!mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        if (sl == 0) TC_TRACE(ti, 0);
+                        if (sl == nslabs - 1) TC_TRACE(ti, 1);
+                        const uint32_t a_dst = tiles_base + (uint32_t)(s * stage_bytes);
+                        if (PAIR) {
+                            // both CTAs report to the barrier of the MMA-issuing CTA
+                            const uint32_t full = mapa_cluster(smem_u32(&sh.full[s]), 0);
+                            mbar_arrive_expect_tx_cluster(full, (uint32_t)stage_bytes);
+                            tma_load_2d_pair(a_dst, &mapA, full, sl * TC_BK, (int)row0);
+                            tma_load_2d_pair(a_dst + TC_A_BYTES, &mapB, full, sl * TC_BK, (int)rank * nb_rows);
+                        } else {
+                            const uint32_t full = smem_u32(&sh.full[s]);
+                            mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
+                            tma_load_2d(a_dst, &mapA, full, sl * TC_BK, (int)row0);
+                            tma_load_2d(a_dst + TC_A_BYTES, &mapB, full, sl * TC_BK, 0);
+                        }
+                    }
+                }
+                if (!ok && rank == 0) {
+                    // give copies that are still in flight a bounded time to land
+                    for (int s = 0; s < nstages; ++s)
+                        for (int tries = 0; tries < 100000; ++tries)
+                            if (mbar_try_wait(smem_u32(&sh.full[s]), 0) || mbar_try_wait(smem_u32(&sh.full[s]), 1)) break;
                 }
             }
-            if (!ok) {
-                // give copies that are still in flight a bounded time to land
-                for (int s = 0; s < TC_STAGES; ++s)
-                    for (int tries = 0; tries < 100000; ++tries)
-                        if (mbar_try_wait(smem_u32(&sh.full[s]), 0) || mbar_try_wait(smem_u32(&sh.full[s]), 1)) break;
-            }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_tf32(p.npad);
-            uint32_t it = 0, ti = 0;
-            bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ti) {
-                const int b = ti & 1;
-                if (!mbar_wait(smem_u32(&sh.tmem_empty[b]), ((ti >> 1) & 1u) ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t acc = tmem_base + (uint32_t)(b * p.npad);
-                for (int sl = 0; sl < nslabs; ++sl, ++it) {
-                    const int s = it % TC_STAGES;
-                    if (!mbar_wait(smem_u32(&sh.full[s]), (it / TC_STAGES) & 1u, abort_flag, p.ctl)) { ok = false; break; }
+        } else if (warp == 1) {
+            // ------------------------------------------------------------ MMA issuer
+            if (lane == 0 && rank == 0) {
+                const uint32_t idesc = make_idesc_tf32(PAIR ? 2 * TC_BM : TC_BM, p.npad);
+                uint32_t it = 0, ti = 0;
+                bool ok = true;
+                for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
+                    const int b = ti & 1;
+                    if (!mbar_wait(smem_u32(&sh.tmem_empty[b]), ((ti >> 1) & 1u) ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = tiles_base + (uint32_t)(s * stage_bytes);
-                    const uint64_t adesc = make_smem_desc(a_addr);
-                    const uint64_t bdesc = make_smem_desc(a_addr + TC_A_BYTES);
+                    const uint32_t acc = tmem_base + (uint32_t)(b * p.npad);
+                    for (int sl = 0; sl < nslabs; ++sl, ++it) {
+                        const int s = it % nstages;
+                        if (!mbar_wait(smem_u32(&sh.full[s]), (it / nstages) & 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        if (sl == 0) TC_TRACE(ti, 2);
+                        if (sl == nslabs - 1) TC_TRACE(ti, 3);
+                        tc_fence_after();
+                        const uint32_t a_addr = tiles_base + (uint32_t)(s * stage_bytes);
+                        const uint64_t adesc = make_smem_desc(a_addr);
+                        const uint64_t bdesc = make_smem_desc(a_addr + TC_A_BYTES);
 #pragma unroll
-                    for (int kk = 0; kk < TC_BK / 8; ++kk)   // 8 tf32 = 32 B per MMA: +2 in 16-byte units
-                        mma_tf32(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&sh.empty[s]));
+                        for (int kk = 0; kk < TC_BK / 8; ++kk) {   // 8 tf32 = 32 B per MMA: +2 in 16-byte units
+                            if (PAIR)
+                                mma_tf32_pair(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
+                            else
+                                mma_tf32(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        // the stage is free (in both CTAs) once these MMAs have read it
+                        if (PAIR) tc_commit_pair(smem_u32(&sh.empty[s])); else tc_commit(smem_u32(&sh.empty[s]));
+                    }
+                    if (ok) {
+                        if (PAIR) tc_commit_pair(smem_u32(&sh.tmem_full[b])); else tc_commit(smem_u32(&sh.tmem_full[b]));
+                    }
                 }
-                if (ok) tc_commit(smem_u32(&sh.tmem_full[b]));
+                // all MMAs issued by this thread have completed once this commit arrives
+                if (PAIR) tc_commit_pair_local(smem_u32(&sh.drain)); else tc_commit(smem_u32(&sh.drain));
+                for (int tries = 0; tries < 4000000; ++tries)
+                    if (mbar_try_wait(smem_u32(&sh.drain), 0)) break;
             }
-            // all MMAs issued by this thread have completed once this commit arrives
-            tc_commit(smem_u32(&sh.drain));
-            for (int tries = 0; tries < 4000000; ++tries)
-                if (mbar_try_wait(smem_u32(&sh.drain), 0)) break;
         }
-    } else {
-        // ------------------------------------------------------------ epilogue
-        const int ew = warp - 2;                  // 0 .. NEPI-1
-        const bool scorer = ew < TC_SCORE_WARPS;
+    } else if (warp < TC_FIRST_STREAM_WARP) {
+        // ------------------------------------------------------------ score warps
+        if (AFFINE) setmaxnreg_dec<TC_REGS_SCORE>();
         const int quarter = warp & 3;             // TMEM lanes this warp may read
         uint32_t ti = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ti) {
+        for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
             const int b = ti & 1;
             const uint32_t ph = (ti >> 1) & 1u;
-            const int64_t row0 = tile * TC_BM;
-            if (scorer) {
-                if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
-                tc_fence_after();
-                float b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F, b4 = CUDART_INF_F;
-                int i1 = 0, i2 = 0, i3 = 0, i4 = 0;
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
-                for (int c = 0; c < p.npad; c += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + (uint32_t)c, v);
+            const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
+            if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
+            tc_fence_after();
+            if (quarter == 0 && lane == 0) TC_TRACE(ti, 4);
+            float b1 = TC_KEY_INIT, b2 = TC_KEY_INIT, b3 = TC_KEY_INIT, b4 = TC_KEY_INIT;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
+            // two register buffers: the next 16 columns are in flight while these are scanned
+            uint32_t ra[16], rb[16];
+            tmem_ld16_issue(taddr, ra);
+            for (int c = 0; c < p.npad; c += 32) {
+                tmem_ld_wait16(ra);
+                tmem_ld16_issue(taddr + (uint32_t)(c + 16), rb);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float sc = fmaf(-2.f, v[j], sh.cn[c + j]);
-                        if (sc < b4) {
-                            const int n = c + j;
-                            if (sc < b3) {
-                                b4 = b3; i4 = i3;
-                                if (sc < b2) {
-                                    b3 = b2; i3 = i2;
-                                    if (sc < b1) { b2 = b1; i2 = i1; b1 = sc; i1 = n; }
-                                    else { b2 = sc; i2 = n; }
-                                } else { b3 = sc; i3 = n; }
-                            } else { b4 = sc; i4 = n; }
-                        }
-                    }
-                }
-                // accumulator buffer b may be overwritten from here on
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh.tmem_empty[b]));
-                const int r = quarter * 32 + lane;
-                if (AFFINE) {
-                    if (!mbar_wait_warp(smem_u32(&sh.lab_empty[b]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
-                    sh.top_score[b][r] = make_float4(b1, b2, b3, b4);
-                    sh.top_idx[b][r] = make_int4(i1, i2, i3, i4);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh.lab_full[b]));
-                } else {
-                    const int64_t row = row0 + r;
-                    if (row < p.N) {
-                        const float e = tc_error_bound(p.D, p.ynorm2[row], cmax2);
-                        p.labels[row] = i1;
-                        tc_decide(p, row, make_float4(b1, b2, b3, b4), make_int4(i1, i2, i3, i4), e);
-                    }
-                }
+                for (int j = 0; j < 16; ++j)
+                    key_insert(make_key(fmaf(-2.f, __uint_as_float(ra[j]), sh.cn[c + j]), c + j), b1, b2, b3, b4);
+                tmem_ld_wait16(rb);
+                if (c + 32 < p.npad) tmem_ld16_issue(taddr + (uint32_t)(c + 32), ra);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    key_insert(make_key(fmaf(-2.f, __uint_as_float(rb[j]), sh.cn[c + 16 + j]), c + 16 + j), b1, b2, b3, b4);
             }
+            if (quarter == 0 && lane == 0) TC_TRACE(ti, 5);
+            // accumulator buffer b may be overwritten from here on
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(mapa_cluster(smem_u32(&sh.tmem_empty[b]), 0));
+                else mbar_arrive(smem_u32(&sh.tmem_empty[b]));
+            }
+            const int r = quarter * 32 + lane;
             if (AFFINE) {
-                if (!mbar_wait_warp(smem_u32(&sh.lab_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
-                const int D4 = p.D >> 2;
-                const float4 *Y4 = reinterpret_cast<const float4 *>(p.Y);
-                const float4 *G4 = reinterpret_cast<const float4 *>(p.gamma);
-                const float4 *B4 = reinterpret_cast<const float4 *>(p.beta);
-                float4 *O4 = reinterpret_cast<float4 *>(p.out);
-                for (int r = ew; r < TC_BM; r += NEPI) {
-                    const int64_t row = row0 + r;
-                    if (row >= p.N) break;
-                    const float4 tsc = sh.top_score[b][r];
-                    const int4 tid4 = sh.top_idx[b][r];
-                    const int l = tid4.x;
-                    const float4 *y4 = Y4 + (size_t)row * D4;
-                    const float4 *g4 = G4 + (size_t)l * D4;
-                    const float4 *b4 = B4 + (size_t)l * D4;
-                    float4 *o4 = O4 + (size_t)row * D4;
-                    if (D4 <= 256) {
-                        float4 res[8];
-                        float ysq = 0.f;
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const int c = lane + 32 * q;
-                            if (c < D4) {
-                                float4 y = __ldcs(y4 + c);
-                                float4 g = __ldg(g4 + c);
-                                float4 bb = __ldg(b4 + c);
-                                ysq = fmaf(y.x, y.x, ysq);
-                                ysq = fmaf(y.y, y.y, ysq);
-                                ysq = fmaf(y.z, y.z, ysq);
-                                ysq = fmaf(y.w, y.w, ysq);
-                                res[q].x = fmaf(g.x, y.x, bb.x);
-                                res[q].y = fmaf(g.y, y.y, bb.y);
-                                res[q].z = fmaf(g.z, y.z, bb.z);
-                                res[q].w = fmaf(g.w, y.w, bb.w);
-                            }
-                        }
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
-                        const float e = tc_error_bound(p.D, ysq, cmax2);
-                        const bool certain = (p.K == 1) || ((tsc.y - tsc.x) > 2.f * e);
-                        if (certain) {
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const int c = lane + 32 * q;
-                                if (c < D4) __stcs(o4 + c, res[q]);
-                            }
-                        }
-                        if (lane == 0) {
-                            p.labels[row] = l;
-                            if (!certain) tc_decide(p, row, tsc, tid4, e);
-                        }
-                    } else {
-                        float ysq = 0.f;
-                        for (int c = lane; c < D4; c += 32) {
-                            float4 y = __ldg(y4 + c);
-                            ysq = fmaf(y.x, y.x, ysq);
-                            ysq = fmaf(y.y, y.y, ysq);
-                            ysq = fmaf(y.z, y.z, ysq);
-                            ysq = fmaf(y.w, y.w, ysq);
-                        }
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
-                        const float e = tc_error_bound(p.D, ysq, cmax2);
-                        const bool certain = (p.K == 1) || ((tsc.y - tsc.x) > 2.f * e);
-                        if (certain) {
-                            for (int c = lane; c < D4; c += 32) {
-                                float4 y = __ldcs(y4 + c);
-                                float4 g = __ldg(g4 + c);
-                                float4 bb = __ldg(b4 + c);
-                                float4 v;
-                                v.x = fmaf(g.x, y.x, bb.x);
-                                v.y = fmaf(g.y, y.y, bb.y);
-                                v.z = fmaf(g.z, y.z, bb.z);
-                                v.w = fmaf(g.w, y.w, bb.w);
-                                __stcs(o4 + c, v);
-                            }
-                        }
-                        if (lane == 0) {
-                            p.labels[row] = l;
-                            if (!certain) tc_decide(p, row, tsc, tid4, e);
-                        }
-                    }
-                }
+                // hand the keys to the streaming warps (buffer b is free once tile ti - 2 is streamed)
+                if (!mbar_wait_warp(smem_u32(&sh.lab_empty[b]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                sh.top_key[b][r] = make_float4(b1, b2, b3, b4);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh.lab_empty[b]));
+                if (lane == 0) mbar_arrive(smem_u32(&sh.lab_full[b]));
+            } else {
+                const int64_t row = row0 + r;
+                if (row < p.N) {
+                    const float e = tc_error_bound(p.D, p.ynorm2[row], cmax2);
+                    p.labels[row] = key_label(b1, p.K);
+                    tc_decide(p, row, make_float4(b1, b2, b3, b4), e);
+                }
             }
+        }
+    } else if (AFFINE) {
+        // ------------------------------------------------------------ streaming warps
+        setmaxnreg_inc<TC_REGS_STREAM>();
+        const int ew = warp - TC_FIRST_STREAM_WARP;
+        uint32_t ti = 0;
+        bool ok = true;
+        for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
+            const int b = ti & 1;
+            const uint32_t ph = (ti >> 1) & 1u;
+            const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
+            if (!mbar_wait_warp(smem_u32(&sh.lab_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
+            if (ew == 0 && lane == 0) TC_TRACE(ti, 6);
+            for (int r = ew; r < TC_BM; r += TC_STREAM_WARPS) {
+                const int64_t row = row0 + r;
+                if (row < p.N) stream_row(p, row, sh.top_key[b][r], cmax2, lane);
+                __syncwarp();
+                if (lane == 0) atomicAdd(&sh.rows_streamed, 1);
+            }
+            __syncwarp();
+            if (ew == 0 && lane == 0) TC_TRACE(ti, 7);
+            if (lane == 0) mbar_arrive(smem_u32(&sh.lab_empty[b]));
         }
     }
 
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync();   // neither CTA's shared memory or TMEM goes away under the other
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+        if (PAIR) tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
+        else tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
 
@@ -554,6 +761,15 @@ bool make_map(CUtensorMap *map, const float *base, int64_t rows, int D, int box_
     return r == CUDA_SUCCESS;
 }
 
+// The affine kernel re-divides its registers among its warpgroups; a division larger than
+// what the block was launched with would wait forever, so it is checked here before launch.
+bool regs_ok(const void *kern)
+{
+    cudaFuncAttributes a{};
+    if (cudaFuncGetAttributes(&a, kern) != cudaSuccess) return false;
+    return (long)a.numRegs * TC_THREADS_AFFINE >= 128L * (TC_REGS_CONTROL + TC_REGS_SCORE + 3 * TC_REGS_STREAM);
+}
+
 int sm_count()
 {
     static int cached[64] = {};
@@ -603,31 +819,77 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     p.N = N;
     p.D = D;
     p.K = K;
-    p.npad = (K + 15) / 16 * 16;
+    p.npad = (K + 31) / 32 * 32;
     int cols = 32;
     while (cols < 2 * p.npad) cols <<= 1;
     p.tmem_cols = cols;
 
-    CUtensorMap mapA, mapB;
-    if (!make_map(&mapA, Y, N, D, TC_BM) || !make_map(&mapB, C, K, D, p.npad)) return cudaErrorInvalidValue;
-
-    const size_t smem = 1024 + (size_t)TC_STAGES * (TC_A_BYTES + (size_t)p.npad * 128) + sizeof(TcShared);
-    const int64_t tiles = (N + TC_BM - 1) / TC_BM;
-    const int sms = sm_count();
-    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     const bool affine = out != nullptr;
-    cudaError_t e;
-    if (affine) {
-        auto kern = assign_tc_kernel<true>;
-        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        kern<<<grid, 32 * (2 + TC_STREAM_WARPS), smem, s>>>(mapA, mapB, p);
-    } else {
-        auto kern = assign_tc_kernel<false>;
-        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        kern<<<grid, 32 * (2 + TC_SCORE_WARPS), smem, s>>>(mapA, mapB, p);
+    // Two CTAs per 256 rows whenever there is more than one tile of rows.
+    const bool pair = N > TC_BM;
+    const int nb_rows = pair ? p.npad / 2 : p.npad;
+    CUtensorMap mapA, mapB;
+    if (!make_map(&mapA, Y, N, D, TC_BM) || !make_map(&mapB, C, K, D, nb_rows)) return cudaErrorInvalidValue;
+
+    const size_t stage_bytes = TC_A_BYTES + (size_t)nb_rows * 128;
+    const size_t smem_budget = 227 * 1024;
+    int stages = (int)((smem_budget - 1024 - sizeof(TcShared)) / stage_bytes);
+    if (stages > TC_MAX_STAGES) stages = TC_MAX_STAGES;
+    if (affine && stages > TC_AFFINE_MAX_STAGES) stages = TC_AFFINE_MAX_STAGES;
+    if (stages < 2) return cudaErrorInvalidValue;
+    p.stages = stages;
+    const size_t smem = 1024 + (size_t)stages * stage_bytes + sizeof(TcShared);
+    // ask for no more shared memory than the kernel uses (the rest of the array serves as L1)
+    const int carveout = (int)((smem * 100 + smem_budget - 1) / smem_budget);
+    const int sms = sm_count();
+    const unsigned threads = affine ? TC_THREADS_AFFINE : TC_THREADS_LABELS;
+    unsigned grid = 1;
+    if (pair) {
+        const int64_t units = (N + 2 * TC_BM - 1) / (2 * TC_BM);
+        const int64_t clusters = units < sms / 2 ? units : sms / 2;
+        grid = (unsigned)(2 * clusters);
     }
+
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = pair ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+
+    cudaError_t e;
+#define CAT_TC_LAUNCH(AFF, PR)                                                                                         \
+    do {                                                                                                               \
+        auto kern = assign_tc_kernel<AFF, PR>;                                                                         \
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)   \
+            return e;                                                                                                  \
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, carveout)) != cudaSuccess) \
+            return e;                                                                                                  \
+        if (AFF && !regs_ok(reinterpret_cast<const void *>(kern))) return cudaErrorLaunchOutOfResources;               \
+        e = cudaLaunchKernelEx(&cfg, kern, mapA, mapB, p);                                                             \
+    } while (0)
+    if (affine) {
+        if (pair) CAT_TC_LAUNCH(true, true); else CAT_TC_LAUNCH(true, false);
+    } else {
+        if (pair) CAT_TC_LAUNCH(false, true); else CAT_TC_LAUNCH(false, false);
+    }
+#undef CAT_TC_LAUNCH
+    if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace cat
+
+#ifdef CAT_TC_TRACE
+extern "C" int cat_tc_trace_read(unsigned long long *host_out)
+{
+    return (int)cudaMemcpyFromSymbol(host_out, cat::g_tc_trace, sizeof(cat::g_tc_trace));
+}
+#endif

@@ -54,12 +54,14 @@ FitWs carve_fit(void *base, int64_t N, int D, int K)
     Carver c(base);
     FitWs w{};
     carve_assign_into(c, w.a, N, D, K);
-    SegGeom g = seg_geometry(N, D, K);
+    SegGeom g = seg_geometry(2 * N, D, 2 * K);   // delta mode is the larger of the two
     size_t KD = (size_t)K * D;
-    w.blk_hist = c.take<uint32_t>((size_t)g.nblk * K);
-    w.cluster_start = c.take<int32_t>((size_t)K + 1);
-    w.seg_start = c.take<int32_t>((size_t)K + 1);
-    w.order = c.take<int32_t>((size_t)N);
+    w.blk_hist = c.take<uint32_t>((size_t)g.nblk * 2 * K);
+    w.key_total = c.take<uint32_t>((size_t)2 * K);
+    w.cluster_start = c.take<int32_t>((size_t)2 * K + 1);
+    w.seg_start = c.take<int32_t>((size_t)2 * K + 1);
+    w.order = c.take<int32_t>((size_t)2 * N);
+    w.labels_prev = c.take<int32_t>((size_t)N);
     w.segpart = c.take<double>((size_t)g.max_segs * 2 * D);
     w.sumQ = c.take<double>(KD);
     w.sumF = c.take<double>(KD);
@@ -114,12 +116,13 @@ static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const fl
     return CAT_OK;
 }
 
-// sort the rows by label: counts, cluster/segment tables and `order` in the workspace
+// sort the rows by label (full mode): counts, cluster/segment tables and `order` in the workspace
 static cat_status_t run_sort(const int32_t *labels, int64_t N, int D, int K, const FitWs &w,
                              int64_t *counts, cudaStream_t s)
 {
     SegGeom g = seg_geometry(N, D, K);
-    CAT_CUDA(launch_label_sort(labels, N, K, g, w.blk_hist, counts, w.cluster_start, w.seg_start, w.order, s));
+    CAT_CUDA(launch_label_sort(labels, nullptr, N, K, g, w.blk_hist, w.key_total, counts, w.cluster_start,
+                               w.seg_start, w.order, s));
     return CAT_OK;
 }
 
@@ -130,7 +133,22 @@ static cat_status_t run_sums(const float *M, int64_t N, int D, int K, const FitW
     SegGeom g = seg_geometry(N, D, K);
     CAT_CUDA(launch_segment_sums(0, M, nullptr, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D, K,
                                  g, w.segpart, s));
-    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, counts, D, K, sums, nullptr, C, s));
+    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, counts, D, K, false, sums, nullptr, C, s));
+    return CAT_OK;
+}
+
+// One centroid update of a Lloyd round from the rows whose label changed: the running sums
+// and sizes in the workspace (sumQ, counts) move by what entered and left each cluster, then
+// c_k = sumQ_k / n_k.  `prev` = all -1 makes every row an entry (the first round).
+static cat_status_t run_delta_update(const float *Yq, const int32_t *labels, const int32_t *prev, int64_t N, int D,
+                                     int K, const FitWs &w, float *C, cudaStream_t s)
+{
+    SegGeom g = seg_geometry(2 * N, D, 2 * K);
+    CAT_CUDA(launch_label_sort(labels, prev, N, K, g, w.blk_hist, w.key_total, w.counts, w.cluster_start,
+                               w.seg_start, w.order, s));
+    CAT_CUDA(launch_segment_sums(0, Yq, nullptr, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D,
+                                 2 * K, g, w.segpart, s));
+    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, true, w.sumQ, nullptr, C, s));
     return CAT_OK;
 }
 
@@ -141,7 +159,7 @@ static cat_status_t run_centred(const float *Yq, const float *Yfp, int64_t N, in
     SegGeom g = seg_geometry(N, D, K);
     CAT_CUDA(launch_segment_sums(2, Yq, Yfp, w.order, w.cluster_start, w.seg_start, meanQ, meanF, D, K, g,
                                  w.segpart, s));
-    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, nullptr, D, K, var, cov, nullptr, s));
+    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, nullptr, D, K, false, var, cov, nullptr, s));
     return CAT_OK;
 }
 
@@ -242,12 +260,19 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
 
     const bool tc = use_tensor_path(N, D, K);
     if (tc) CAT_CUDA(launch_row_norms(Yq, N, D, w.a.ynorm2, s));   // Yq is fixed: once per fit
+
+    // Lloyd rounds.  Two label buffers alternate so that a round sees the previous round's
+    // labels and the final assignment lands in `labels`; the running per-cluster sums and
+    // sizes start at zero with "no previous label" (-1) for every row.
+    int32_t *lab[2] = {labels, w.labels_prev};
+    CAT_CUDA(cudaMemsetAsync(lab[(iters & 1) ^ 1], 0xFF, (size_t)N * sizeof(int32_t), s));
+    CAT_CUDA(cudaMemsetAsync(w.sumQ, 0, KD * sizeof(double), s));
+    CAT_CUDA(cudaMemsetAsync(w.counts, 0, (size_t)K * sizeof(int64_t), s));
     for (int t = 0; t < iters; ++t) {
-        st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false);
+        int32_t *cur = lab[(iters - t) & 1], *prev = lab[((iters - t) & 1) ^ 1];
+        st = run_assign(Yq, N, D, K, C, cur, w.a, nullptr, nullptr, nullptr, s, tc, false);
         if (st != CAT_OK) return st;
-        st = run_sort(labels, N, D, K, w, w.counts, s);
-        if (st != CAT_OK) return st;
-        st = run_sums(Yq, N, D, K, w, w.counts, w.sumQ, C, s);   // sums -> centroid update
+        st = run_delta_update(Yq, cur, prev, N, D, K, w, C, s);
         if (st != CAT_OK) return st;
     }
 
@@ -260,7 +285,7 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
         SegGeom g = seg_geometry(N, D, K);
         CAT_CUDA(launch_segment_sums(1, Yq, Yfp, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D,
                                      K, g, w.segpart, s));
-        CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, w.sumQ, w.sumF, nullptr, s));
+        CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, false, w.sumQ, w.sumF, nullptr, s));
     }
     CAT_CUDA(launch_means_from_sums(w.sumQ, w.counts, D, K, meanQ, s));
     CAT_CUDA(launch_means_from_sums(w.sumF, w.counts, D, K, meanF, s));

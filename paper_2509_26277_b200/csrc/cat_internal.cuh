@@ -36,14 +36,15 @@ struct Control {
     int64_t pad[4];
 };
 
-// Geometry of the sort-based segmented sums for one (N, D, K): identical in the workspace
-// query and at launch time.
+// Geometry of the sort-based segmented sums for NE entries over KK keys (full mode: N rows,
+// K labels; delta mode: 2N virtual entries, 2K keys): identical in the workspace query and
+// at launch time.
 struct SegGeom {
-    int nblk;       // 1024-row blocks of the label sort
+    int nblk;       // 1024-entry blocks of the sort
     int seg_rows;   // rows per segment (multiple of 128)
-    int max_segs;   // upper bound on the number of segments: ceil(N / seg_rows) + K
+    int max_segs;   // upper bound on the number of segments: ceil(NE / seg_rows) + KK
 };
-SegGeom seg_geometry(int64_t N, int D, int K);
+SegGeom seg_geometry(int64_t NE, int D, int KK);
 
 struct AssignWs {          // what assign/apply need
     Control *ctl;
@@ -61,10 +62,13 @@ AssignWs carve_assign(void *base, int64_t N, int D, int K);
 
 struct FitWs {
     AssignWs a;
-    uint32_t *blk_hist;    // [nblk][K] label histogram / offsets of the sort
-    int32_t *cluster_start; // [K+1] first position of each cluster in `order`
-    int32_t *seg_start;    // [K+1] first segment of each cluster
-    int32_t *order;        // [N] row indices sorted by label (stable)
+    // sized for delta mode (2N virtual entries, 2K keys)
+    uint32_t *blk_hist;    // [nblk][2K] key histogram / offsets of the sort
+    uint32_t *key_total;   // [2K] entries per key
+    int32_t *cluster_start; // [2K+1] first position of each key in `order`
+    int32_t *seg_start;    // [2K+1] first segment of each key
+    int32_t *order;        // [2N] row indices sorted by key (stable)
+    int32_t *labels_prev;  // [N] labels of the previous Lloyd round
     double *segpart;       // [max_segs][2][D] per-segment partial sums
     double *sumQ, *sumF, *var, *cov;   // [K*D] each
     double *meanQ, *meanF;             // [K*D] each
@@ -105,23 +109,27 @@ cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, co
                                      const uint64_t *cand_list, Control *ctl, const float *gamma,
                                      const float *beta, float *out, cudaStream_t s);
 
-// Stable sort of the row indices by label: counts[K], cluster_start[K+1], seg_start[K+1], order[N].
-// Labels outside [0, K) are left out.
-cudaError_t launch_label_sort(const int32_t *labels, int64_t N, int K, const SegGeom &g, uint32_t *blk_hist,
-                              int64_t *counts, int32_t *cluster_start, int32_t *seg_start, int32_t *order,
-                              cudaStream_t s);
+// Stable sort of the row indices by key.  prev == NULL (full mode): key = label, counts[k] = size of
+// cluster k.  prev != NULL (delta mode): entries only for rows with labels[i] != prev[i], under keys
+// labels[i] and K + prev[i]; counts[k] += (rows that entered k) - (rows that left k).  Tables have one
+// entry per key (+1).  Labels outside [0, K) are left out.
+cudaError_t launch_label_sort(const int32_t *labels, const int32_t *prev, int64_t N, int K, const SegGeom &g,
+                              uint32_t *blk_hist, uint32_t *key_total, int64_t *counts, int32_t *cluster_start,
+                              int32_t *seg_start, int32_t *order, cudaStream_t s);
 
-// Per-segment partial sums.  mode 0: column sums of Yq (plane 0); mode 1: of Yq and Yf (planes 0, 1);
-// mode 2: centred moments sum (q-muQ)^2 (plane 0) and sum (q-muQ)(f-muF) (plane 1).
+// Per-segment partial sums over KK keys.  mode 0: column sums of Yq (plane 0); mode 1: of Yq and Yf
+// (planes 0, 1); mode 2 (full mode only): centred moments sum (q-muQ)^2 (plane 0) and
+// sum (q-muQ)(f-muF) (plane 1).
 cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, const int32_t *order,
                                 const int32_t *cluster_start, const int32_t *seg_start, const double *meanQ,
-                                const double *meanF, int D, int K, const SegGeom &g, double *part,
+                                const double *meanF, int D, int KK, const SegGeom &g, double *part,
                                 cudaStream_t s);
 
-// Adds each cluster's segment partials in order into out0 (and out1 if not NULL); with C also
-// writes the centroid float(out0 / n_k) for clusters with n_k > 0.
+// Adds each cluster's segment partials in order into out0 (and out1 if not NULL); in delta mode
+// out0[k] += (partials of key k) - (partials of key K + k).  With C also writes the centroid
+// float(out0 / n_k) for clusters with n_k > 0.
 cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
-                                   int K, double *out0, double *out1, float *C, cudaStream_t s);
+                                   int K, bool delta, double *out0, double *out1, float *C, cudaStream_t s);
 
 cudaError_t launch_centroids_from_sums(const double *sums, const int64_t *counts, int D, int K,
                                        float *C, cudaStream_t s);

@@ -1,9 +1,17 @@
 // Segmented (per-cluster) sums through a stable sort of the rows by label.
 //
-//   label_hist_kernel     per-block label histograms (1024 rows per block)
-//   label_scan_kernel     cluster sizes, cluster offsets, per-block offsets, segment table
+//   label_hist_kernel     per-block key histograms (1024 entries per block)
+//   label_scan_blocks_kernel / label_scan_keys_kernel
+//                         per-block offsets, key totals, key offsets, segment table, cluster sizes
 //   label_scatter_kernel  stable scatter of the row indices: order[] lists the rows of
-//                         cluster 0 in ascending row order, then cluster 1, ...
+//                         key 0 in ascending row order, then key 1, ...
+//
+// Two modes.  Full: every row is an entry with key = its label (K keys).  Delta (the Lloyd
+// rounds of cat_fit): only rows whose label differs from the previous round's are entries,
+// each twice -- under key `new label` (its values enter that cluster's sum) and under key
+// K + `old label` (they leave that one) -- so 2K keys over 2N virtual entries, nearly all of
+// them empty once the clustering settles.  The running sums S_k += sum(in) - sum(out) are the
+// same per-cluster sums up to fp64 rounding, at the cost of the rows that moved.
 //   segment_sums_kernel   one CTA per segment (<= seg_rows consecutive entries of order[], all of
 //                         one cluster): streams those rows with 128-bit loads and keeps the
 //                         column sums in fp64 registers -- no atomics, no shared accumulators,
@@ -23,90 +31,143 @@ namespace {
 constexpr int SORT_BLOCK = 1024;     // rows per histogram / scatter block
 constexpr int SEG_THREADS = 256;
 
-__global__ void __launch_bounds__(SORT_BLOCK) label_hist_kernel(const int32_t *__restrict__ labels, int64_t N,
-                                                                 int K, uint32_t *__restrict__ blk_hist)
+// Key of virtual entry e: entries [0, N) are the rows under their current label; in delta
+// mode (prev != NULL) a row whose label did not change has no entry, and entries [N, 2N)
+// are the changed rows under K + previous label.  -1 = no entry.
+__device__ __forceinline__ int entry_key(const int32_t *__restrict__ cur, const int32_t *__restrict__ prev,
+                                         int64_t N, int K, int64_t e)
 {
-    extern __shared__ uint32_t hist[];   // [K]
-    for (int k = threadIdx.x; k < K; k += SORT_BLOCK) hist[k] = 0;
-    __syncthreads();
-    const int64_t row = (int64_t)blockIdx.x * SORT_BLOCK + threadIdx.x;
-    if (row < N) {
-        const int l = labels[row];
-        if (l >= 0 && l < K) atomicAdd(&hist[l], 1u);
+    if (e < N) {
+        const int l = cur[e];
+        if (l < 0 || l >= K) return -1;
+        if (prev && prev[e] == l) return -1;
+        return l;
     }
-    __syncthreads();
-    for (int k = threadIdx.x; k < K; k += SORT_BLOCK) blk_hist[(size_t)blockIdx.x * K + k] = hist[k];
+    if (!prev || e >= 2 * N) return -1;
+    const int64_t r = e - N;
+    const int o = prev[r];
+    if (o < 0 || o >= K || o == cur[r]) return -1;
+    return K + o;
 }
 
-// One CTA.  Thread k walks the blocks of cluster k: blk_hist[b][k] becomes the number of rows
-// of cluster k in blocks before b.  Then cluster_start (exclusive scan of the sizes) and
-// seg_start (exclusive scan of ceil(size / seg_rows)), each with K + 1 entries.
-__global__ void __launch_bounds__(512) label_scan_kernel(uint32_t *__restrict__ blk_hist, int nblk, int K,
-                                                         int seg_rows, int64_t *__restrict__ counts,
-                                                         int32_t *__restrict__ cluster_start,
-                                                         int32_t *__restrict__ seg_start)
+__global__ void __launch_bounds__(SORT_BLOCK) label_hist_kernel(const int32_t *__restrict__ cur,
+                                                                 const int32_t *__restrict__ prev, int64_t N, int K,
+                                                                 int KK, uint32_t *__restrict__ blk_hist)
 {
-    __shared__ uint32_t size_s[CAT_MAX_K];
-    const int k = threadIdx.x;
-    uint32_t run = 0;
+    extern __shared__ uint32_t hist[];   // [KK]
+    for (int k = threadIdx.x; k < KK; k += SORT_BLOCK) hist[k] = 0;
+    __syncthreads();
+    const int64_t e = (int64_t)blockIdx.x * SORT_BLOCK + threadIdx.x;
+    const int l = entry_key(cur, prev, N, K, e);
+    if (l >= 0) atomicAdd(&hist[l], 1u);
+    __syncthreads();
+    for (int k = threadIdx.x; k < KK; k += SORT_BLOCK) blk_hist[(size_t)blockIdx.x * KK + k] = hist[k];
+}
+
+// One warp per key: blk_hist[b][k] becomes the number of entries of key k in blocks before
+// b, key_total[k] their total.
+__global__ void __launch_bounds__(256) label_scan_blocks_kernel(uint32_t *__restrict__ blk_hist, int nblk, int KK,
+                                                                 uint32_t *__restrict__ key_total)
+{
+    const int k = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (k >= KK) return;
+    uint32_t carry = 0;
+    for (int b0 = 0; b0 < nblk; b0 += 32) {
+        const int b = b0 + lane;
+        const uint32_t v = (b < nblk) ? blk_hist[(size_t)b * KK + k] : 0u;
+        uint32_t incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (b < nblk) blk_hist[(size_t)b * KK + k] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) key_total[k] = carry;
+}
+
+// One CTA of 1024 threads (KK <= 1024): exclusive scans of the key totals (cluster_start) and
+// of the segment counts ceil(total / seg_rows) (seg_start), KK + 1 entries each; cluster sizes:
+// full mode counts[k] = total[k]; delta mode counts[k] += total[k] - total[K + k].
+__global__ void __launch_bounds__(1024) label_scan_keys_kernel(const uint32_t *__restrict__ key_total, int K, int KK,
+                                                                int seg_rows, int delta, int64_t *__restrict__ counts,
+                                                                int32_t *__restrict__ cluster_start,
+                                                                int32_t *__restrict__ seg_start)
+{
+    __shared__ uint32_t wsum_a[32], wsum_s[32];
+    const int k = threadIdx.x, lane = k & 31, w = k >> 5;
+    const uint32_t tot = (k < KK) ? key_total[k] : 0u;
+    const uint32_t sg = (tot + (uint32_t)seg_rows - 1) / (uint32_t)seg_rows;
+    uint32_t ia = tot, is = sg;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o);
+        const uint32_t ts = __shfl_up_sync(0xffffffffu, is, o);
+        if (lane >= o) { ia += ta; is += ts; }
+    }
+    if (lane == 31) { wsum_a[w] = ia; wsum_s[w] = is; }
+    __syncthreads();
+    if (w == 0) {
+        uint32_t a = wsum_a[lane], sgs = wsum_s[lane];
+        uint32_t xa = a, xs = sgs;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t ta = __shfl_up_sync(0xffffffffu, xa, o);
+            const uint32_t ts = __shfl_up_sync(0xffffffffu, xs, o);
+            if (lane >= o) { xa += ta; xs += ts; }
+        }
+        wsum_a[lane] = xa - a;   // exclusive
+        wsum_s[lane] = xs - sgs;
+    }
+    __syncthreads();
+    const uint32_t ea = wsum_a[w] + ia - tot, es = wsum_s[w] + is - sg;
+    if (k < KK) {
+        cluster_start[k] = (int32_t)ea;
+        seg_start[k] = (int32_t)es;
+        if (k == KK - 1) {
+            cluster_start[KK] = (int32_t)(ea + tot);
+            seg_start[KK] = (int32_t)(es + sg);
+        }
+    }
     if (k < K) {
-        for (int b = 0; b < nblk; ++b) {
-            const size_t o = (size_t)b * K + k;
-            const uint32_t v = blk_hist[o];
-            blk_hist[o] = run;
-            run += v;
-        }
-        counts[k] = (int64_t)run;
-        size_s[k] = run;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t a = 0, sgs = 0;
-        for (int q = 0; q < K; ++q) {
-            cluster_start[q] = (int32_t)a;
-            seg_start[q] = (int32_t)sgs;
-            a += size_s[q];
-            sgs += (size_s[q] + (uint32_t)seg_rows - 1) / (uint32_t)seg_rows;
-        }
-        cluster_start[K] = (int32_t)a;
-        seg_start[K] = (int32_t)sgs;
+        if (delta) counts[k] += (int64_t)tot - (int64_t)key_total[K + k];
+        else counts[k] = (int64_t)tot;
     }
 }
 
-// Stable scatter.  Within a block, a row's rank among the rows of its cluster is
-// (rows of that cluster in earlier warps) + (rows of that cluster in earlier lanes).
-__global__ void __launch_bounds__(SORT_BLOCK) label_scatter_kernel(const int32_t *__restrict__ labels, int64_t N,
-                                                                    int K, const uint32_t *__restrict__ blk_hist,
+// Stable scatter.  Within a block, an entry's rank among the entries of its key is
+// (entries of that key in earlier warps) + (entries of that key in earlier lanes).
+__global__ void __launch_bounds__(SORT_BLOCK) label_scatter_kernel(const int32_t *__restrict__ cur,
+                                                                    const int32_t *__restrict__ prev, int64_t N, int K,
+                                                                    int KK, const uint32_t *__restrict__ blk_hist,
                                                                     const int32_t *__restrict__ cluster_start,
                                                                     int32_t *__restrict__ order)
 {
-    extern __shared__ uint16_t warp_hist[];   // [32][K]
+    extern __shared__ uint16_t warp_hist[];   // [32][KK]
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    for (int e = tid; e < 32 * K; e += SORT_BLOCK) warp_hist[e] = 0;
+    for (int e = tid; e < 32 * KK; e += SORT_BLOCK) warp_hist[e] = 0;
     __syncthreads();
-    const int64_t row = (int64_t)blockIdx.x * SORT_BLOCK + tid;
-    int l = -1;
-    if (row < N) {
-        l = labels[row];
-        if (l < 0 || l >= K) l = -1;
-    }
+    const int64_t e = (int64_t)blockIdx.x * SORT_BLOCK + tid;
+    const int l = entry_key(cur, prev, N, K, e);
     const unsigned peers = __match_any_sync(0xffffffffu, l);
     const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
-    if (l >= 0 && rank_in_warp == 0) warp_hist[w * K + l] = (uint16_t)__popc(peers);
+    if (l >= 0 && rank_in_warp == 0) warp_hist[w * KK + l] = (uint16_t)__popc(peers);
     __syncthreads();
-    for (int k = tid; k < K; k += SORT_BLOCK) {
+    for (int k = tid; k < KK; k += SORT_BLOCK) {
         uint16_t run = 0;
         for (int q = 0; q < 32; ++q) {
-            const uint16_t v = warp_hist[q * K + k];
-            warp_hist[q * K + k] = run;
+            const uint16_t v = warp_hist[q * KK + k];
+            warp_hist[q * KK + k] = run;
             run = (uint16_t)(run + v);
         }
     }
     __syncthreads();
     if (l >= 0) {
-        const uint32_t pos = (uint32_t)cluster_start[l] + blk_hist[(size_t)blockIdx.x * K + l] +
-                             warp_hist[w * K + l] + (uint32_t)rank_in_warp;
-        order[pos] = (int32_t)row;
+        const uint32_t pos = (uint32_t)cluster_start[l] + blk_hist[(size_t)blockIdx.x * KK + l] +
+                             warp_hist[w * KK + l] + (uint32_t)rank_in_warp;
+        order[pos] = (int32_t)(e < N ? e : e - N);
     }
 }
 
@@ -266,10 +327,11 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
     }
 }
 
-// out0/out1[k*D+j] = sum over the segments of cluster k of plane 0/1 (out1 may be NULL);
-// with C != NULL also C[k*D+j] = float(out0 / n_k) where n_k > 0.
+// out0/out1[k*D+j] = sum over the segments of key k of plane 0/1 (out1 may be NULL); in
+// delta mode out0[k*D+j] += (segments of key k) - (segments of key K + k).  With C != NULL
+// also C[k*D+j] = float(out0 / n_k) where n_k > 0.
 __global__ void segment_combine_kernel(const double *__restrict__ part, const int32_t *__restrict__ seg_start,
-                                       const int64_t *__restrict__ counts, int D, size_t KD,
+                                       const int64_t *__restrict__ counts, int D, int K, size_t KD, int delta,
                                        double *__restrict__ out0, double *__restrict__ out1,
                                        float *__restrict__ C)
 {
@@ -282,6 +344,11 @@ __global__ void segment_combine_kernel(const double *__restrict__ part, const in
     for (int sgm = s0; sgm < s1; ++sgm) {
         a += part[((size_t)sgm * 2) * D + j];
         if (out1) b += part[((size_t)sgm * 2 + 1) * D + j];
+    }
+    if (delta) {
+        double m = 0.0;
+        for (int sgm = seg_start[K + k]; sgm < seg_start[K + k + 1]; ++sgm) m += part[((size_t)sgm * 2) * D + j];
+        a = out0[e] + (a - m);
     }
     out0[e] = a;
     if (out1) out1[e] = b;
@@ -300,28 +367,37 @@ int tpr_for(int units)
 
 }  // namespace
 
-SegGeom seg_geometry(int64_t N, int D, int K)
+// Geometry for NE virtual entries over KK keys.
+SegGeom seg_geometry(int64_t NE, int D, int KK)
 {
     SegGeom g{};
-    g.nblk = (int)((N + SORT_BLOCK - 1) / SORT_BLOCK);
-    int64_t sr = (N + 2047) / 2048;
+    g.nblk = (int)((NE + SORT_BLOCK - 1) / SORT_BLOCK);
+    int64_t sr = (NE + 2047) / 2048;
     if (sr < 128) sr = 128;
     sr = (sr + 127) / 128 * 128;
     g.seg_rows = (int)sr;
-    g.max_segs = (int)((N + sr - 1) / sr) + K;
+    g.max_segs = (int)((NE + sr - 1) / sr) + KK;
     (void)D;
     return g;
 }
 
-cudaError_t launch_label_sort(const int32_t *labels, int64_t N, int K, const SegGeom &g, uint32_t *blk_hist,
-                              int64_t *counts, int32_t *cluster_start, int32_t *seg_start, int32_t *order,
-                              cudaStream_t s)
+cudaError_t launch_label_sort(const int32_t *labels, const int32_t *prev, int64_t N, int K, const SegGeom &g,
+                              uint32_t *blk_hist, uint32_t *key_total, int64_t *counts, int32_t *cluster_start,
+                              int32_t *seg_start, int32_t *order, cudaStream_t s)
 {
-    label_hist_kernel<<<g.nblk, SORT_BLOCK, (size_t)K * sizeof(uint32_t), s>>>(labels, N, K, blk_hist);
-    label_scan_kernel<<<1, 512, 0, s>>>(blk_hist, g.nblk, K, g.seg_rows, counts, cluster_start, seg_start);
-    label_scatter_kernel<<<g.nblk, SORT_BLOCK, (size_t)32 * K * sizeof(uint16_t), s>>>(labels, N, K, blk_hist,
-                                                                                       cluster_start, order);
-    count_launch(3);
+    const int KK = prev ? 2 * K : K;
+    label_hist_kernel<<<g.nblk, SORT_BLOCK, (size_t)KK * sizeof(uint32_t), s>>>(labels, prev, N, K, KK, blk_hist);
+    label_scan_blocks_kernel<<<(KK * 32 + 255) / 256, 256, 0, s>>>(blk_hist, g.nblk, KK, key_total);
+    label_scan_keys_kernel<<<1, 1024, 0, s>>>(key_total, K, KK, g.seg_rows, prev ? 1 : 0, counts, cluster_start,
+                                               seg_start);
+    const size_t sc_smem = (size_t)32 * KK * sizeof(uint16_t);
+    if (sc_smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(label_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)sc_smem);
+        if (e != cudaSuccess) return e;
+    }
+    label_scatter_kernel<<<g.nblk, SORT_BLOCK, sc_smem, s>>>(labels, prev, N, K, KK, blk_hist, cluster_start, order);
+    count_launch(4);
     return cudaGetLastError();
 }
 
@@ -366,12 +442,12 @@ cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, cons
 }
 
 cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
-                                   int K, double *out0, double *out1, float *C, cudaStream_t s)
+                                   int K, bool delta, double *out0, double *out1, float *C, cudaStream_t s)
 {
     const size_t KD = (size_t)K * D;
     const int threads = 256;
     const unsigned blocks = (unsigned)((KD + threads - 1) / threads);
-    segment_combine_kernel<<<blocks, threads, 0, s>>>(part, seg_start, counts, D, KD, out0, out1, C);
+    segment_combine_kernel<<<blocks, threads, 0, s>>>(part, seg_start, counts, D, K, KD, delta ? 1 : 0, out0, out1, C);
     count_launch();
     return cudaGetLastError();
 }

@@ -540,20 +540,33 @@ __global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
         if (row < 0 || row >= N) continue;
         int cand[4];
         const float *cp[4];
+        int ncand = 0;   // the list is filled from the front: unused slots are at the end
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             int k = (int)((packed >> (16 * q)) & 0xFFFFu);
             cand[q] = (k < K) ? k : -1;
             cp[q] = C + (size_t)(k < K ? k : 0) * D;
+            if (k < K) ncand = q + 1;
         }
         const float *y = Y + (size_t)row * D;
         double s[4] = {0.0, 0.0, 0.0, 0.0};
-        for (int j = lane; j < D; j += 32) {
-            const double yv = (double)y[j];
+        if (ncand <= 2) {
+            // the common case: only the two nearest are in question
+            for (int j = lane; j < D; j += 32) {
+                const double yv = (double)y[j];
+                const double d0 = yv - (double)cp[0][j];
+                const double d1 = yv - (double)cp[1][j];
+                s[0] = fma(d0, d0, s[0]);
+                s[1] = fma(d1, d1, s[1]);
+            }
+        } else {
+            for (int j = lane; j < D; j += 32) {
+                const double yv = (double)y[j];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const double d = yv - (double)cp[q][j];
-                s[q] = fma(d, d, s[q]);
+                for (int q = 0; q < 4; ++q) {
+                    const double d = yv - (double)cp[q][j];
+                    s[q] = fma(d, d, s[q]);
+                }
             }
         }
         double best = CUDART_INF;

@@ -38,10 +38,12 @@ namespace {
 constexpr int TC_BM = 128;                   // rows per CTA tile (UMMA M per CTA)
 constexpr int TC_BK = 32;                    // fp32 per slab = 128 B = one swizzle row
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 4;  // 16 KB
-constexpr int TC_MAX_STAGES = 8;
+constexpr int TC_MAX_A_STAGES = 8;           // ring of row slabs (filled from HBM: deep)
+constexpr int TC_MAX_B_STAGES = 4;           // ring of centroid slabs (filled from L2: shallow)
 constexpr uint64_t TC_TIMEOUT_NS = 2000000000ull;
 
-// Warp roles.  Warp 0: TMA producer, warp 1: MMA issuer (2, 3 idle), warps 4-7: score warps
+// Warp roles.  Warp 0: TMA producer of the row slabs, warp 1: MMA issuer, warp 2: TMA producer
+// of the centroid slabs (warp 3 idle), warps 4-7: score warps
 // (TMEM lane quarter = warp & 3); with the affine epilogue also warps 8-19: streaming warps.
 constexpr int TC_FIRST_SCORE_WARP = 4;
 constexpr int TC_SCORE_WARPS = 4;
@@ -62,8 +64,9 @@ static_assert(128 * (TC_REGS_CONTROL + TC_REGS_SCORE + 3 * TC_REGS_STREAM) <= TC
 // The streaming warps read through L1, and the number of loads an SM keeps in flight shrinks
 // with L1: a shared-memory carve-out of 200 KB and more costs a third of the streaming rate
 // (measured), about 100 KB costs nothing.  The tile period of the affine kernel is long
-// enough for a shallow TMA ring, so that kernel takes the smaller carve-out.
-constexpr int TC_AFFINE_MAX_STAGES = 3;
+// enough for shallow TMA rings, so that kernel takes the smaller carve-out.
+constexpr int TC_AFFINE_A_STAGES = 4;
+constexpr int TC_AFFINE_B_STAGES = 2;
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -330,12 +333,15 @@ struct TcParams {
     int K;
     int npad;       // K rounded up to 32 (the score warps read TMEM 32 columns per step)
     int tmem_cols;  // power of two >= 2 * npad
-    int stages;     // shared-memory pipeline stages (<= TC_MAX_STAGES)
+    int a_stages;   // ring depths (<= TC_MAX_A_STAGES, TC_MAX_B_STAGES)
+    int b_stages;
 };
 
 struct TcShared {
-    uint64_t full[TC_MAX_STAGES];
-    uint64_t empty[TC_MAX_STAGES];
+    uint64_t a_full[TC_MAX_A_STAGES];
+    uint64_t a_empty[TC_MAX_A_STAGES];
+    uint64_t b_full[TC_MAX_B_STAGES];
+    uint64_t b_empty[TC_MAX_B_STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t lab_full[2];
@@ -472,9 +478,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;
     unsigned char *tiles = smem_raw + (tiles_base - raw);
     const int nb_rows = PAIR ? (p.npad >> 1) : p.npad;   // centroid rows this CTA stages per slab
-    const int stage_bytes = TC_A_BYTES + nb_rows * 128;
-    const int nstages = p.stages;
-    TcShared &sh = *reinterpret_cast<TcShared *>(tiles + (size_t)nstages * stage_bytes);
+    const int b_bytes = nb_rows * 128;
+    const int na = p.a_stages, nb = p.b_stages;
+    const uint32_t b_base = tiles_base + (uint32_t)(na * TC_A_BYTES);   // the centroid ring follows the row ring
+    TcShared &sh = *reinterpret_cast<TcShared *>(tiles + (size_t)na * TC_A_BYTES + (size_t)nb * b_bytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // 0 = the CTA that issues the MMAs
@@ -486,9 +493,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const int nslabs = (p.D + TC_BK - 1) / TC_BK;
 
     if (tid == 0) {
-        for (int s = 0; s < nstages; ++s) {
-            mbar_init(smem_u32(&sh.full[s]), PAIR ? 2 : 1);    // one expect_tx arrival per CTA
-            mbar_init(smem_u32(&sh.empty[s]), 1);
+        for (int s = 0; s < na; ++s) {
+            mbar_init(smem_u32(&sh.a_full[s]), PAIR ? 2 : 1);    // one expect_tx arrival per CTA
+            mbar_init(smem_u32(&sh.a_empty[s]), 1);
+        }
+        for (int s = 0; s < nb; ++s) {
+            mbar_init(smem_u32(&sh.b_full[s]), PAIR ? 2 : 1);
+            mbar_init(smem_u32(&sh.b_empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sh.tmem_full[b]), 1);
@@ -546,31 +557,57 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         if (!wait_progress(&sh.rows_streamed, (int)(ti - 1) * TC_BM, abort_flag, p.ctl)) { ok = false; break; }
                     }
                     for (int sl = 0; sl < nslabs; ++sl, ++it) {
-                        const int s = it % nstages;
-                        const uint32_t ph = (it / nstages) & 1u;
-                        if (!mbar_wait(smem_u32(&sh.empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        const int s = it % na;
+                        const uint32_t ph = (it / na) & 1u;
+                        if (!mbar_wait(smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
                         if (sl == 0) TC_TRACE(ti, 0);
                         if (sl == nslabs - 1) TC_TRACE(ti, 1);
-                        const uint32_t a_dst = tiles_base + (uint32_t)(s * stage_bytes);
+                        const uint32_t a_dst = tiles_base + (uint32_t)(s * TC_A_BYTES);
                         if (PAIR) {
                             // both CTAs report to the barrier of the MMA-issuing CTA
-                            const uint32_t full = mapa_cluster(smem_u32(&sh.full[s]), 0);
-                            mbar_arrive_expect_tx_cluster(full, (uint32_t)stage_bytes);
+                            const uint32_t full = mapa_cluster(smem_u32(&sh.a_full[s]), 0);
+                            mbar_arrive_expect_tx_cluster(full, (uint32_t)TC_A_BYTES);
                             tma_load_2d_pair(a_dst, &mapA, full, sl * TC_BK, (int)row0);
-                            tma_load_2d_pair(a_dst + TC_A_BYTES, &mapB, full, sl * TC_BK, (int)rank * nb_rows);
                         } else {
-                            const uint32_t full = smem_u32(&sh.full[s]);
-                            mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
+                            const uint32_t full = smem_u32(&sh.a_full[s]);
+                            mbar_arrive_expect_tx(full, (uint32_t)TC_A_BYTES);
                             tma_load_2d(a_dst, &mapA, full, sl * TC_BK, (int)row0);
-                            tma_load_2d(a_dst + TC_A_BYTES, &mapB, full, sl * TC_BK, 0);
                         }
                     }
                 }
                 if (!ok && rank == 0) {
                     // give copies that are still in flight a bounded time to land
-                    for (int s = 0; s < nstages; ++s)
+                    for (int s = 0; s < na; ++s)
                         for (int tries = 0; tries < 100000; ++tries)
-                            if (mbar_try_wait(smem_u32(&sh.full[s]), 0) || mbar_try_wait(smem_u32(&sh.full[s]), 1)) break;
+                            if (mbar_try_wait(smem_u32(&sh.a_full[s]), 0) || mbar_try_wait(smem_u32(&sh.a_full[s]), 1)) break;
+                }
+            }
+        } else if (warp == 2) {
+            // ------------------------------------------------------------ TMA producer, centroid slabs
+            if (lane == 0) {
+                uint32_t it = 0;
+                bool ok = true;
+                for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step) {
+                    for (int sl = 0; sl < nslabs; ++sl, ++it) {
+                        const int s = it % nb;
+                        const uint32_t ph = (it / nb) & 1u;
+                        if (!mbar_wait(smem_u32(&sh.b_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        const uint32_t b_dst = b_base + (uint32_t)(s * b_bytes);
+                        if (PAIR) {
+                            const uint32_t full = mapa_cluster(smem_u32(&sh.b_full[s]), 0);
+                            mbar_arrive_expect_tx_cluster(full, (uint32_t)b_bytes);
+                            tma_load_2d_pair(b_dst, &mapB, full, sl * TC_BK, (int)rank * nb_rows);
+                        } else {
+                            const uint32_t full = smem_u32(&sh.b_full[s]);
+                            mbar_arrive_expect_tx(full, (uint32_t)b_bytes);
+                            tma_load_2d(b_dst, &mapB, full, sl * TC_BK, 0);
+                        }
+                    }
+                }
+                if (!ok && rank == 0) {
+                    for (int s = 0; s < nb; ++s)
+                        for (int tries = 0; tries < 100000; ++tries)
+                            if (mbar_try_wait(smem_u32(&sh.b_full[s]), 0) || mbar_try_wait(smem_u32(&sh.b_full[s]), 1)) break;
                 }
             }
         } else if (warp == 1) {
@@ -585,14 +622,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     tc_fence_after();
                     const uint32_t acc = tmem_base + (uint32_t)(b * p.npad);
                     for (int sl = 0; sl < nslabs; ++sl, ++it) {
-                        const int s = it % nstages;
-                        if (!mbar_wait(smem_u32(&sh.full[s]), (it / nstages) & 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        const int sa = it % na, sb = it % nb;
+                        if (!mbar_wait(smem_u32(&sh.b_full[sb]), (it / nb) & 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        if (!mbar_wait(smem_u32(&sh.a_full[sa]), (it / na) & 1u, abort_flag, p.ctl)) { ok = false; break; }
                         if (sl == 0) TC_TRACE(ti, 2);
                         if (sl == nslabs - 1) TC_TRACE(ti, 3);
                         tc_fence_after();
-                        const uint32_t a_addr = tiles_base + (uint32_t)(s * stage_bytes);
-                        const uint64_t adesc = make_smem_desc(a_addr);
-                        const uint64_t bdesc = make_smem_desc(a_addr + TC_A_BYTES);
+                        const uint64_t adesc = make_smem_desc(tiles_base + (uint32_t)(sa * TC_A_BYTES));
+                        const uint64_t bdesc = make_smem_desc(b_base + (uint32_t)(sb * b_bytes));
 #pragma unroll
                         for (int kk = 0; kk < TC_BK / 8; ++kk) {   // 8 tf32 = 32 B per MMA: +2 in 16-byte units
                             if (PAIR)
@@ -600,8 +637,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                             else
                                 mma_tf32(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
                         }
-                        // the stage is free (in both CTAs) once these MMAs have read it
-                        if (PAIR) tc_commit_pair(smem_u32(&sh.empty[s])); else tc_commit(smem_u32(&sh.empty[s]));
+                        // both slabs are free (in both CTAs) once these MMAs have read them
+                        if (PAIR) {
+                            tc_commit_pair(smem_u32(&sh.a_empty[sa]));
+                            tc_commit_pair(smem_u32(&sh.b_empty[sb]));
+                        } else {
+                            tc_commit(smem_u32(&sh.a_empty[sa]));
+                            tc_commit(smem_u32(&sh.b_empty[sb]));
+                        }
                     }
                     if (ok) {
                         if (PAIR) tc_commit_pair(smem_u32(&sh.tmem_full[b])); else tc_commit(smem_u32(&sh.tmem_full[b]));
@@ -831,14 +874,17 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     CUtensorMap mapA, mapB;
     if (!make_map(&mapA, Y, N, D, TC_BM) || !make_map(&mapB, C, K, D, nb_rows)) return cudaErrorInvalidValue;
 
-    const size_t stage_bytes = TC_A_BYTES + (size_t)nb_rows * 128;
+    // ring depths: the centroid ring is shallow (its slabs come out of L2), the row ring takes the rest
+    const size_t b_bytes = (size_t)nb_rows * 128;
     const size_t smem_budget = 227 * 1024;
-    int stages = (int)((smem_budget - 1024 - sizeof(TcShared)) / stage_bytes);
-    if (stages > TC_MAX_STAGES) stages = TC_MAX_STAGES;
-    if (affine && stages > TC_AFFINE_MAX_STAGES) stages = TC_AFFINE_MAX_STAGES;
-    if (stages < 2) return cudaErrorInvalidValue;
-    p.stages = stages;
-    const size_t smem = 1024 + (size_t)stages * stage_bytes + sizeof(TcShared);
+    int b_stages = affine ? TC_AFFINE_B_STAGES : 3;
+    int a_stages = (int)((smem_budget - 1024 - sizeof(TcShared) - b_stages * b_bytes) / TC_A_BYTES);
+    if (a_stages > TC_MAX_A_STAGES) a_stages = TC_MAX_A_STAGES;
+    if (affine && a_stages > TC_AFFINE_A_STAGES) a_stages = TC_AFFINE_A_STAGES;
+    if (a_stages < 2) return cudaErrorInvalidValue;
+    p.a_stages = a_stages;
+    p.b_stages = b_stages;
+    const size_t smem = 1024 + (size_t)a_stages * TC_A_BYTES + (size_t)b_stages * b_bytes + sizeof(TcShared);
     // ask for no more shared memory than the kernel uses (the rest of the array serves as L1)
     const int carveout = (int)((smem * 100 + smem_budget - 1) / smem_budget);
     const int sms = sm_count();

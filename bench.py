@@ -299,10 +299,10 @@ def run_cuda(args):
             "fit_s_per_lloyd_iter": lloyd_ms * 1e-3,
             "fit_ms": fit_ms_step, "apply_ms": apply_ms_step,
             "wall_s": t_wall,
-            "roofline": {"bound": "hbm", "kernel": "assign_kernel<AFFINE> (cat_apply)",
+            "roofline": {"bound": "hbm", "kernel": "assign_tc_kernel<affine, pair> (the one kernel of cat_apply besides the exact pass)",
                          "achieved": apply_gbs, "peak": peak, "unit": "GB/s", "frac": apply_gbs / peak,
                          "peak_source": peak_src, "traffic": None},
-            "roofline_fit": {"bound": "hbm", "kernel": "one Lloyd round of cat_fit (assign + segmented sums)",
+            "roofline_fit": {"bound": "hbm", "kernel": "one Lloyd round of cat_fit (assign_tc_kernel<labels, pair> + exact pass + delta centroid update)",
                              "achieved": lloyd_gbs, "peak": peak, "unit": "GB/s", "frac": lloyd_gbs / peak},
             "exact_pass_rows": {"apply": rep_apply["refined_rows_last"],
                                 "fit_all_assignments": rep_fit["refined_rows_total"] if rep_fit else None},

@@ -79,8 +79,12 @@ typedef struct cat_fit_diag {
  * labels_out    [N] out, may be NULL.
  * init_centroids [K, D] in, may be NULL; must not alias centroids_out.
  * diag          device pointer to one cat_fit_diag_t, may be NULL.
- * Labels are decided in fp64 whenever the fast fp32 scores cannot separate
- * the two nearest centroids; sums and moments are accumulated in fp64.
+ * Labels are decided in fp64 whenever the fast scores cannot separate the two
+ * nearest centroids; sums and moments are accumulated in fp64.  In the Lloyd
+ * rounds the per-cluster sums are carried from round to round and updated with
+ * the rows whose label changed (the same sums up to fp64 rounding).
+ * The workspace holds, besides tables of a few N and K*D words, an fp16 copy
+ * of Yq (N*D*2 bytes) that the tensor-core assignment reads in every round.
  */
 size_t cat_fit_workspace_bytes(int64_t N, int32_t D, int32_t K);
 

@@ -63,6 +63,9 @@ FitWs carve_fit(void *base, int64_t N, int D, int K)
     w.order = c.take<int32_t>((size_t)2 * N);
     w.labels_prev = c.take<int32_t>((size_t)N);
     w.segpart = c.take<double>((size_t)g.max_segs * 2 * D);
+    w.yh = c.take<uint16_t>((size_t)N * D);
+    w.ch = c.take<uint16_t>(KD);
+    w.hscale = c.take<float>(4);
     w.sumQ = c.take<double>(KD);
     w.sumF = c.take<double>(KD);
     w.var = c.take<double>(KD);
@@ -100,13 +103,15 @@ static bool use_tensor_path(int64_t N, int D, int K)
 static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const float *C,
                                int32_t *labels, const AssignWs &w, const float *gamma,
                                const float *beta, float *out, cudaStream_t s,
-                               bool row_norms_ready = false, bool top_level = true)
+                               bool row_norms_ready = false, bool top_level = true,
+                               const void *Yh = nullptr, void *Ch = nullptr, const float *hscale = nullptr)
 {
     CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s, top_level));
     if (use_tensor_path(N, D, K)) {
         if (!out && !row_norms_ready) CAT_CUDA(launch_row_norms(Y, N, D, w.ynorm2, s));
+        if (Yh) CAT_CUDA(launch_to_half(C, (size_t)K * D, hscale, Ch, s));
         CAT_CUDA(launch_assign_tc(Y, N, D, K, C, w.cnorm, w.ynorm2, labels, w.refine_rows, w.cand_rows,
-                                  w.cand_list, w.ctl, gamma, beta, out, s));
+                                  w.cand_list, w.ctl, gamma, beta, out, s, Yh, Ch, hscale));
         CAT_CUDA(launch_refine_candidates(Y, N, D, K, C, labels, w.cand_rows, w.cand_list, w.ctl, gamma,
                                           beta, out, s));
     } else {
@@ -259,7 +264,14 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
                              cudaMemcpyDeviceToDevice, s));
 
     const bool tc = use_tensor_path(N, D, K);
-    if (tc) CAT_CUDA(launch_row_norms(Yq, N, D, w.a.ynorm2, s));   // Yq is fixed: once per fit
+    // Yq is fixed over the fit: its row norms, and where the shape allows an fp16 copy for the
+    // tensor cores, are made once
+    // (only with the default start: centroids that are rows or means of rows cannot exceed the
+    // largest magnitude of Yq, which sets the fp16 scale; caller-provided ones could overflow it)
+    const bool half = tc && !init_centroids && tc_half_supported(N, D, K);
+    const void *Yh = half ? w.yh : nullptr;
+    if (half) CAT_CUDA(launch_half_shadow(Yq, N, D, w.a.ynorm2, w.hscale, w.yh, s));
+    else if (tc) CAT_CUDA(launch_row_norms(Yq, N, D, w.a.ynorm2, s));
 
     // Lloyd rounds.  Two label buffers alternate so that a round sees the previous round's
     // labels and the final assignment lands in `labels`; the running per-cluster sums and
@@ -270,14 +282,14 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     CAT_CUDA(cudaMemsetAsync(w.counts, 0, (size_t)K * sizeof(int64_t), s));
     for (int t = 0; t < iters; ++t) {
         int32_t *cur = lab[(iters - t) & 1], *prev = lab[((iters - t) & 1) ^ 1];
-        st = run_assign(Yq, N, D, K, C, cur, w.a, nullptr, nullptr, nullptr, s, tc, false);
+        st = run_assign(Yq, N, D, K, C, cur, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale);
         if (st != CAT_OK) return st;
         st = run_delta_update(Yq, cur, prev, N, D, K, w, C, s);
         if (st != CAT_OK) return st;
     }
 
     // final assignment, then the closed form
-    st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false);
+    st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale);
     if (st != CAT_OK) return st;
     st = run_sort(labels, N, D, K, w, w.counts, s);
     if (st != CAT_OK) return st;

@@ -70,6 +70,9 @@ struct FitWs {
     int32_t *order;        // [2N] row indices sorted by key (stable)
     int32_t *labels_prev;  // [N] labels of the previous Lloyd round
     double *segpart;       // [max_segs][2][D] per-segment partial sums
+    void *yh;              // [N*D] fp16 copy of Yq (tensor-core fits with D % 8 == 0)
+    void *ch;              // [K*D] fp16 copy of the centroids
+    float *hscale;         // [4] scale of the fp16 copies
     double *sumQ, *sumF, *var, *cov;   // [K*D] each
     double *meanQ, *meanF;             // [K*D] each
     int64_t *counts;       // [K]
@@ -98,10 +101,20 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
 // Tensor-core (tcgen05, TF32) variant of launch_assign; ynorm2 is needed when out == nullptr.
 bool tc_supported(int64_t N, int D, int K);
 cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaStream_t s);
+// With Yh / Ch / scale (labels only): the fp16 copies of the rows and centroids are the MMA operands.
 cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,
                              const float *ynorm2, int32_t *labels, int32_t *refine_rows,
                              int32_t *cand_rows, uint64_t *cand_list, Control *ctl,
-                             const float *gamma, const float *beta, float *out, cudaStream_t s);
+                             const float *gamma, const float *beta, float *out, cudaStream_t s,
+                             const void *Yh = nullptr, const void *Ch = nullptr, const float *scale = nullptr);
+
+// fp16 copy of a matrix for repeated assignments: squared row norms, scale[4] (power-of-two scale,
+// -2 / scale^2, subnormal rounding error) and Yh = fp16(Y * scale).  Needs D % 8 == 0.
+bool tc_half_supported(int64_t N, int D, int K);
+cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, float *scale, void *Yh,
+                               cudaStream_t s);
+// dst = fp16(src * scale[0]) for n elements (n % 4 == 0)
+cudaError_t launch_to_half(const float *src, size_t n, const float *scale, void *dst, cudaStream_t s);
 
 // Exact fp64 decision among the listed candidates of each queued row; optional affine output.
 cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, const float *C,

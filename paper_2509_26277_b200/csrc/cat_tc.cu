@@ -17,6 +17,13 @@
 // tensor core taken as <= 2^-22 per term; the last term is the index packed into the
 // key).  Rows it cannot decide go to the same exact fp64 pass, so labels stay exact.
 //
+// cat_fit assigns the same rows many times, so it keeps an fp16 copy of them (scaled by a
+// power of two so that the largest magnitude sits near 2^14, rounded to nearest) and runs the
+// labels kernel on that copy with kind::f16: twice the MMA rate of TF32, half the row bytes,
+// and a tighter operand bound (2^-11 per operand instead of 2^-10):
+//     e <= (2^-9 + (2D+2) 2^-22) ||y|| cmax + 2 a sqrt(D) (||y|| + cmax) + 2 D a^2 + 4 u cmax^2 + (packing term)
+// where a = 2^-25 / scale is the absolute rounding error of an element in fp16's subnormal range.
+//
 // For inference, streaming warps then read every row of the tile once more and write
 // gamma_l * y + beta_l for the fast label l; an undecided row is queued and the exact pass
 // rewrites its output.  The TMA producer may run at most one tile ahead of the streaming
@@ -29,6 +36,7 @@
 #include "cat_internal.cuh"
 
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <math_constants.h>
 
 namespace cat {
@@ -36,8 +44,8 @@ namespace cat {
 namespace {
 
 constexpr int TC_BM = 128;                   // rows per CTA tile (UMMA M per CTA)
-constexpr int TC_BK = 32;                    // fp32 per slab = 128 B = one swizzle row
-constexpr int TC_A_BYTES = TC_BM * TC_BK * 4;  // 16 KB
+constexpr int TC_SLAB_BYTES = 128;           // bytes of a row per slab = one swizzle row (32 fp32 or 64 fp16)
+constexpr int TC_A_BYTES = TC_BM * TC_SLAB_BYTES;  // 16 KB
 constexpr int TC_MAX_A_STAGES = 8;           // ring of row slabs (filled from HBM: deep)
 constexpr int TC_MAX_B_STAGES = 4;           // ring of centroid slabs (filled from L2: shallow)
 constexpr uint64_t TC_TIMEOUT_NS = 2000000000ull;
@@ -254,6 +262,25 @@ __device__ __forceinline__ void mma_tf32_pair(uint32_t tmem_d, uint64_t adesc, u
         : "memory");
 }
 
+__device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_f16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -296,10 +323,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr)
     return d;
 }
 
-// D = F32, A = B = TF32, both K-major, M = m (128, or 256 over a CTA pair), N = n.
-__host__ __device__ constexpr uint32_t make_idesc_tf32(int m, int n)
+// D = F32, A and B of one type (fmt 2 = TF32, 0 = F16), both K-major, M = m (128, or 256 over a
+// CTA pair), N = n.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n, uint32_t fmt)
 {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // Optional timeline of the first two CTAs (compiled in only with -DCAT_TC_TRACE): globaltimer
@@ -320,6 +348,7 @@ struct TcParams {
     const float *Y;
     const float *cnorm;
     const float *ynorm2;   // [N] squared row norms (labels-only mode)
+    const float *scale;    // fp16 operands: {scale, -2 / scale^2, 2^-25 / scale} in device memory
     int32_t *labels;
     int32_t *refine_rows;
     int32_t *cand_rows;    // rows whose exact decision only needs the listed candidates
@@ -388,6 +417,18 @@ __device__ __forceinline__ float tc_error_bound(int D, float ysq, float cmax2)
     const float pk = 3.0517578e-5f;                                         // 2^-15: index packed into the key
     const float yc = sqrtf(ysq) * sqrtf(cmax2);
     return 1.0625f * ((a + 2.f * pk) * yc + (4.f * u + pk) * cmax2);
+}
+
+// Same for fp16 operands (round to nearest, scaled by a power of two; a = absolute rounding
+// error of an element that falls into fp16's subnormal range).
+__device__ __forceinline__ float tc_error_bound_half(int D, float ysq, float cmax2, float a)
+{
+    const float u = 5.9604645e-8f;   // 2^-24
+    const float r = 1.953125e-3f * 1.001f + (2.f * (float)D + 2.f) * 2.3841858e-7f;  // 2^-9 (1 + 2^-12) + (2D+2) 2^-22
+    const float pk = 3.0517578e-5f;
+    const float yn = sqrtf(ysq), cn = sqrtf(cmax2);
+    return 1.0625f * ((r + 2.f * pk) * yn * cn + 2.f * a * sqrtf((float)D) * (yn + cn) + 2.f * (float)D * a * a +
+                      (4.f * u + pk) * cmax2);
 }
 
 // Decision for one row from its four smallest keys.  Returns true when the fast argmin is
@@ -468,7 +509,8 @@ __device__ __forceinline__ void stream_row(const TcParams &p, int64_t row, float
 // loads the slabs of its own 128 rows and of HALF the centroids; the MMA (M = 256, issued
 // by the CTA of rank 0) reads both halves, and each CTA finds the scores of its own rows in
 // its own TMEM.
-template <bool AFFINE, bool PAIR>
+// HALF: operands are the fp16 copies of the rows and centroids (64 columns per slab, kind::f16).
+template <bool AFFINE, bool PAIR, bool HALF>
 __global__ void __launch_bounds__(AFFINE ? TC_THREADS_AFFINE : TC_THREADS_LABELS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p)
 {
@@ -490,7 +532,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const int64_t num_units = PAIR ? (p.N + 2 * TC_BM - 1) / (2 * TC_BM) : (p.N + TC_BM - 1) / TC_BM;
     const int64_t unit_first = PAIR ? (int64_t)(blockIdx.x >> 1) : (int64_t)blockIdx.x;
     const int64_t unit_step = PAIR ? (int64_t)(gridDim.x >> 1) : (int64_t)gridDim.x;
-    const int nslabs = (p.D + TC_BK - 1) / TC_BK;
+    constexpr int BK = HALF ? 64 : 32;   // columns per slab
+    const int nslabs = (p.D + BK - 1) / BK;
+    const float coef = HALF ? p.scale[1] : -2.f;               // score = cn + coef * accumulator
+    const float abs_err = HALF ? p.scale[2] : 0.f;
 
     if (tid == 0) {
         for (int s = 0; s < na; ++s) {
@@ -567,11 +612,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                             // both CTAs report to the barrier of the MMA-issuing CTA
                             const uint32_t full = mapa_cluster(smem_u32(&sh.a_full[s]), 0);
                             mbar_arrive_expect_tx_cluster(full, (uint32_t)TC_A_BYTES);
-                            tma_load_2d_pair(a_dst, &mapA, full, sl * TC_BK, (int)row0);
+                            tma_load_2d_pair(a_dst, &mapA, full, sl * BK, (int)row0);
                         } else {
                             const uint32_t full = smem_u32(&sh.a_full[s]);
                             mbar_arrive_expect_tx(full, (uint32_t)TC_A_BYTES);
-                            tma_load_2d(a_dst, &mapA, full, sl * TC_BK, (int)row0);
+                            tma_load_2d(a_dst, &mapA, full, sl * BK, (int)row0);
                         }
                     }
                 }
@@ -596,11 +641,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         if (PAIR) {
                             const uint32_t full = mapa_cluster(smem_u32(&sh.b_full[s]), 0);
                             mbar_arrive_expect_tx_cluster(full, (uint32_t)b_bytes);
-                            tma_load_2d_pair(b_dst, &mapB, full, sl * TC_BK, (int)rank * nb_rows);
+                            tma_load_2d_pair(b_dst, &mapB, full, sl * BK, (int)rank * nb_rows);
                         } else {
                             const uint32_t full = smem_u32(&sh.b_full[s]);
                             mbar_arrive_expect_tx(full, (uint32_t)b_bytes);
-                            tma_load_2d(b_dst, &mapB, full, sl * TC_BK, 0);
+                            tma_load_2d(b_dst, &mapB, full, sl * BK, 0);
                         }
                     }
                 }
@@ -613,7 +658,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         } else if (warp == 1) {
             // ------------------------------------------------------------ MMA issuer
             if (lane == 0 && rank == 0) {
-                const uint32_t idesc = make_idesc_tf32(PAIR ? 2 * TC_BM : TC_BM, p.npad);
+                const uint32_t idesc = make_idesc(PAIR ? 2 * TC_BM : TC_BM, p.npad, HALF ? 0u : 2u);
                 uint32_t it = 0, ti = 0;
                 bool ok = true;
                 for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
@@ -631,11 +676,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         const uint64_t adesc = make_smem_desc(tiles_base + (uint32_t)(sa * TC_A_BYTES));
                         const uint64_t bdesc = make_smem_desc(b_base + (uint32_t)(sb * b_bytes));
 #pragma unroll
-                        for (int kk = 0; kk < TC_BK / 8; ++kk) {   // 8 tf32 = 32 B per MMA: +2 in 16-byte units
-                            if (PAIR)
-                                mma_tf32_pair(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
-                            else
-                                mma_tf32(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < 4; ++kk) {   // 8 tf32 or 16 f16 = 32 B per MMA: +2 in 16-byte units
+                            const uint32_t accum = (sl > 0 || kk > 0) ? 1u : 0u;
+                            if (HALF) {
+                                if (PAIR) mma_f16_pair(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, accum);
+                                else mma_f16(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, accum);
+                            } else {
+                                if (PAIR) mma_tf32_pair(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, accum);
+                                else mma_tf32(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, accum);
+                            }
                         }
                         // both slabs are free (in both CTAs) once these MMAs have read them
                         if (PAIR) {
@@ -679,12 +728,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 tmem_ld16_issue(taddr + (uint32_t)(c + 16), rb);
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    key_insert(make_key(fmaf(-2.f, __uint_as_float(ra[j]), sh.cn[c + j]), c + j), b1, b2, b3, b4);
+                    key_insert(make_key(fmaf(coef, __uint_as_float(ra[j]), sh.cn[c + j]), c + j), b1, b2, b3, b4);
                 tmem_ld_wait16(rb);
                 if (c + 32 < p.npad) tmem_ld16_issue(taddr + (uint32_t)(c + 32), ra);
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    key_insert(make_key(fmaf(-2.f, __uint_as_float(rb[j]), sh.cn[c + 16 + j]), c + 16 + j), b1, b2, b3, b4);
+                    key_insert(make_key(fmaf(coef, __uint_as_float(rb[j]), sh.cn[c + 16 + j]), c + 16 + j), b1, b2, b3, b4);
             }
             if (quarter == 0 && lane == 0) TC_TRACE(ti, 5);
             // accumulator buffer b may be overwritten from here on
@@ -704,7 +753,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             } else {
                 const int64_t row = row0 + r;
                 if (row < p.N) {
-                    const float e = tc_error_bound(p.D, p.ynorm2[row], cmax2);
+                    const float e = HALF ? tc_error_bound_half(p.D, p.ynorm2[row], cmax2, abs_err)
+                                         : tc_error_bound(p.D, p.ynorm2[row], cmax2);
                     p.labels[row] = key_label(b1, p.K);
                     tc_decide(p, row, make_float4(b1, b2, b3, b4), e);
                 }
@@ -767,6 +817,69 @@ __global__ void row_norms_kernel(const float *__restrict__ Y, int64_t N, int D, 
     if (lane == 0) out[row] = s * 1.0001f;
 }
 
+// Squared row norms as above, and the largest magnitude of the matrix (as the bits of a
+// non-negative float, which order like unsigned integers) into scale_bits[0].
+__global__ void row_norms_amax_kernel(const float *__restrict__ Y, int64_t N, int D, float *__restrict__ out,
+                                      unsigned int *__restrict__ amax_bits)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (row >= N) return;
+    const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)row * D);
+    float s = 0.f, m = 0.f;
+    for (int c = lane; c < (D >> 2); c += 32) {
+        float4 v = __ldg(y4 + c);
+        s = fmaf(v.x, v.x, s);
+        s = fmaf(v.y, v.y, s);
+        s = fmaf(v.z, v.z, s);
+        s = fmaf(v.w, v.w, s);
+        m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, o);
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    }
+    if (lane == 0) {
+        out[row] = s * 1.0001f;
+        if (m == m && m < CUDART_INF_F) atomicMax(amax_bits, __float_as_uint(m));
+    }
+}
+
+// scale[0] = power of two that brings the largest magnitude to [2^13, 2^14); scale[1] = -2 / scale^2
+// (turns the fp16 accumulator into -2 y.c); scale[2] = 2^-25 / scale (rounding error, in the units
+// of the data, of an element that lands in fp16's subnormal range).
+__global__ void half_scale_kernel(float *scale)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const float amax = __uint_as_float(reinterpret_cast<unsigned int *>(scale)[0]);
+    int e = 0;
+    if (amax > 0.f) frexpf(amax, &e);    // amax = f * 2^e, f in [0.5, 1)
+    int sh = 14 - e;
+    if (sh > 100) sh = 100;
+    if (sh < -100) sh = -100;
+    const float sc = ldexpf(1.f, sh);
+    scale[0] = sc;
+    scale[1] = -2.f / (sc * sc);
+    scale[2] = 2.9802322e-8f / sc;
+}
+
+// dst = fp16(src * scale[0]), round to nearest; n4 = number of float4 groups
+__global__ void to_half_kernel(const float4 *__restrict__ src, size_t n4, const float *__restrict__ scale,
+                               uint2 *__restrict__ dst)
+{
+    const float sc = scale[0];
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const float4 v = __ldcs(src + i);
+        const __half2 lo = __floats2half2_rn(v.x * sc, v.y * sc);
+        const __half2 hi = __floats2half2_rn(v.z * sc, v.w * sc);
+        uint2 o;
+        o.x = *reinterpret_cast<const unsigned int *>(&lo);
+        o.y = *reinterpret_cast<const unsigned int *>(&hi);
+        dst[i] = o;
+    }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -788,17 +901,19 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// 2-D fp32 row-major [rows, D] viewed in boxes of box_rows x 32 columns, 128-byte swizzle,
-// zero fill outside the matrix.
-bool make_map(CUtensorMap *map, const float *base, int64_t rows, int D, int box_rows)
+// 2-D row-major [rows, D] of fp32 (or fp16) viewed in boxes of box_rows x 128 bytes, 128-byte
+// swizzle, zero fill outside the matrix.
+bool make_map(CUtensorMap *map, const void *base, bool half, int64_t rows, int D, int box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
+    const size_t esz = half ? 2 : 4;
     cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)D * sizeof(float)};
-    cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+    cuuint64_t strides[1] = {(cuuint64_t)D * esz};
+    cuuint32_t box[2] = {(cuuint32_t)(TC_SLAB_BYTES / esz), (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, estr,
+    CUresult r = fn(map, half ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                    const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
@@ -842,10 +957,47 @@ cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaS
     return cudaGetLastError();
 }
 
+cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, float *scale, void *Yh,
+                               cudaStream_t s)
+{
+    cudaError_t e = cudaMemsetAsync(scale, 0, 4 * sizeof(float), s);
+    if (e != cudaSuccess) return e;
+    const int threads = 256;
+    const int64_t blocks = (N * 32 + threads - 1) / threads;
+    row_norms_amax_kernel<<<(unsigned)blocks, threads, 0, s>>>(Y, N, D, ynorm2, reinterpret_cast<unsigned int *>(scale));
+    half_scale_kernel<<<1, 32, 0, s>>>(scale);
+    const size_t n4 = (size_t)N * D / 4;
+    size_t cb = (n4 + threads - 1) / threads;
+    if (cb > (size_t)sm_count() * 16) cb = (size_t)sm_count() * 16;
+    to_half_kernel<<<(unsigned)cb, threads, 0, s>>>(reinterpret_cast<const float4 *>(Y), n4, scale,
+                                                    reinterpret_cast<uint2 *>(Yh));
+    count_launch(3);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_to_half(const float *src, size_t n, const float *scale, void *dst, cudaStream_t s)
+{
+    const int threads = 256;
+    const size_t n4 = n / 4;
+    size_t cb = (n4 + threads - 1) / threads;
+    if (cb > (size_t)sm_count() * 16) cb = (size_t)sm_count() * 16;
+    if (cb < 1) cb = 1;
+    to_half_kernel<<<(unsigned)cb, threads, 0, s>>>(reinterpret_cast<const float4 *>(src), n4, scale,
+                                                    reinterpret_cast<uint2 *>(dst));
+    count_launch();
+    return cudaGetLastError();
+}
+
+bool tc_half_supported(int64_t N, int D, int K)
+{
+    return tc_supported(N, D, K) && (D % 8 == 0);
+}
+
 cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,
                              const float *ynorm2, int32_t *labels, int32_t *refine_rows,
                              int32_t *cand_rows, uint64_t *cand_list, Control *ctl,
-                             const float *gamma, const float *beta, float *out, cudaStream_t s)
+                             const float *gamma, const float *beta, float *out, cudaStream_t s,
+                             const void *Yh, const void *Ch, const float *scale)
 {
     TcParams p{};
     p.Y = Y;
@@ -868,11 +1020,19 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     p.tmem_cols = cols;
 
     const bool affine = out != nullptr;
+    const bool half = (Yh != nullptr) && !affine;
+    p.scale = scale;
     // Two CTAs per 256 rows whenever there is more than one tile of rows.
     const bool pair = N > TC_BM;
     const int nb_rows = pair ? p.npad / 2 : p.npad;
     CUtensorMap mapA, mapB;
-    if (!make_map(&mapA, Y, N, D, TC_BM) || !make_map(&mapB, C, K, D, nb_rows)) return cudaErrorInvalidValue;
+    if (half) {
+        if (!make_map(&mapA, Yh, true, N, D, TC_BM) || !make_map(&mapB, Ch, true, K, D, nb_rows))
+            return cudaErrorInvalidValue;
+    } else {
+        if (!make_map(&mapA, Y, false, N, D, TC_BM) || !make_map(&mapB, C, false, K, D, nb_rows))
+            return cudaErrorInvalidValue;
+    }
 
     // ring depths: the centroid ring is shallow (its slabs come out of L2), the row ring takes the rest
     const size_t b_bytes = (size_t)nb_rows * 128;
@@ -910,9 +1070,9 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     cfg.numAttrs = 1;
 
     cudaError_t e;
-#define CAT_TC_LAUNCH(AFF, PR)                                                                                         \
+#define CAT_TC_LAUNCH(AFF, PR, HF)                                                                                      \
     do {                                                                                                               \
-        auto kern = assign_tc_kernel<AFF, PR>;                                                                         \
+        auto kern = assign_tc_kernel<AFF, PR, HF>;                                                                      \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)   \
             return e;                                                                                                  \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, carveout)) != cudaSuccess) \
@@ -921,9 +1081,11 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
         e = cudaLaunchKernelEx(&cfg, kern, mapA, mapB, p);                                                             \
     } while (0)
     if (affine) {
-        if (pair) CAT_TC_LAUNCH(true, true); else CAT_TC_LAUNCH(true, false);
+        if (pair) CAT_TC_LAUNCH(true, true, false); else CAT_TC_LAUNCH(true, false, false);
+    } else if (half) {
+        if (pair) CAT_TC_LAUNCH(false, true, true); else CAT_TC_LAUNCH(false, false, true);
     } else {
-        if (pair) CAT_TC_LAUNCH(false, true); else CAT_TC_LAUNCH(false, false);
+        if (pair) CAT_TC_LAUNCH(false, true, false); else CAT_TC_LAUNCH(false, false, false);
     }
 #undef CAT_TC_LAUNCH
     if (e != cudaSuccess) return e;

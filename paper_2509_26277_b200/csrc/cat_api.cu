@@ -104,12 +104,15 @@ static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const fl
                                int32_t *labels, const AssignWs &w, const float *gamma,
                                const float *beta, float *out, cudaStream_t s,
                                bool row_norms_ready = false, bool top_level = true,
-                               const void *Yh = nullptr, void *Ch = nullptr, const float *hscale = nullptr)
+                               const void *Yh = nullptr, void *Ch = nullptr, const float *hscale = nullptr,
+                               bool centroids_ready = false)
 {
-    CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s, top_level));
+    // centroids_ready: the centroid update that produced C has already left its norms, its fp16
+    // copy and empty exact-pass queues in the workspace
+    if (!centroids_ready) CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s, top_level));
     if (use_tensor_path(N, D, K)) {
         if (!out && !row_norms_ready) CAT_CUDA(launch_row_norms(Y, N, D, w.ynorm2, s));
-        if (Yh) CAT_CUDA(launch_to_half(C, (size_t)K * D, hscale, Ch, s));
+        if (Yh && !centroids_ready) CAT_CUDA(launch_to_half(C, (size_t)K * D, hscale, Ch, s));
         CAT_CUDA(launch_assign_tc(Y, N, D, K, C, w.cnorm, w.ynorm2, labels, w.refine_rows, w.cand_rows,
                                   w.cand_list, w.ctl, gamma, beta, out, s, Yh, Ch, hscale));
         CAT_CUDA(launch_refine_candidates(Y, N, D, K, C, labels, w.cand_rows, w.cand_list, w.ctl, gamma,
@@ -146,14 +149,15 @@ static cat_status_t run_sums(const float *M, int64_t N, int D, int K, const FitW
 // and sizes in the workspace (sumQ, counts) move by what entered and left each cluster, then
 // c_k = sumQ_k / n_k.  `prev` = all -1 makes every row an entry (the first round).
 static cat_status_t run_delta_update(const float *Yq, const int32_t *labels, const int32_t *prev, int64_t N, int D,
-                                     int K, const FitWs &w, float *C, cudaStream_t s)
+                                     int K, const FitWs &w, float *C, bool half, cudaStream_t s)
 {
     SegGeom g = seg_geometry(2 * N, D, 2 * K);
     CAT_CUDA(launch_label_sort(labels, prev, N, K, g, w.blk_hist, w.key_total, w.counts, w.cluster_start,
                                w.seg_start, w.order, s));
     CAT_CUDA(launch_segment_sums(0, Yq, nullptr, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D,
                                  2 * K, g, w.segpart, s));
-    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, true, w.sumQ, nullptr, C, s));
+    CAT_CUDA(launch_centroid_update(w.segpart, w.seg_start, w.counts, D, K, w.sumQ, C, w.a.cnorm, w.hscale,
+                                    half ? w.ch : nullptr, w.a.ctl, s));
     return CAT_OK;
 }
 
@@ -282,14 +286,16 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     CAT_CUDA(cudaMemsetAsync(w.counts, 0, (size_t)K * sizeof(int64_t), s));
     for (int t = 0; t < iters; ++t) {
         int32_t *cur = lab[(iters - t) & 1], *prev = lab[((iters - t) & 1) ^ 1];
-        st = run_assign(Yq, N, D, K, C, cur, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale);
+        st = run_assign(Yq, N, D, K, C, cur, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale,
+                        t > 0);
         if (st != CAT_OK) return st;
-        st = run_delta_update(Yq, cur, prev, N, D, K, w, C, s);
+        st = run_delta_update(Yq, cur, prev, N, D, K, w, C, half, s);
         if (st != CAT_OK) return st;
     }
 
     // final assignment, then the closed form
-    st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale);
+    st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale,
+                    iters > 0);
     if (st != CAT_OK) return st;
     st = run_sort(labels, N, D, K, w, w.counts, s);
     if (st != CAT_OK) return st;

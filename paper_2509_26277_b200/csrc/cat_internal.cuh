@@ -144,6 +144,12 @@ cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, cons
 cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
                                    int K, bool delta, double *out0, double *out1, float *C, cudaStream_t s);
 
+// Delta-mode centroid update fused with what the next assignment needs: running sums, centroids,
+// their squared norms, (with Ch) their fp16 copy, and the reset of the exact-pass queues.
+cudaError_t launch_centroid_update(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
+                                   int K, double *sums, float *C, float *cnorm, const float *scale, void *Ch,
+                                   Control *ctl, cudaStream_t s);
+
 cudaError_t launch_centroids_from_sums(const double *sums, const int64_t *counts, int D, int K,
                                        float *C, cudaStream_t s);
 cudaError_t launch_means_from_sums(const double *sums, const int64_t *counts, int D, int K,

@@ -24,6 +24,8 @@
 // sum (q - muQ)^2, sum (q - muQ)(f - muF) with the cluster means held in registers.
 #include "cat_internal.cuh"
 
+#include <cuda_fp16.h>
+
 namespace cat {
 
 namespace {
@@ -61,10 +63,10 @@ __global__ void __launch_bounds__(SORT_BLOCK) label_hist_kernel(const int32_t *_
     const int l = entry_key(cur, prev, N, K, e);
     if (l >= 0) atomicAdd(&hist[l], 1u);
     __syncthreads();
-    for (int k = threadIdx.x; k < KK; k += SORT_BLOCK) blk_hist[(size_t)blockIdx.x * KK + k] = hist[k];
+    for (int k = threadIdx.x; k < KK; k += SORT_BLOCK) blk_hist[(size_t)k * gridDim.x + blockIdx.x] = hist[k];   // [key][block]
 }
 
-// One warp per key: blk_hist[b][k] becomes the number of entries of key k in blocks before
+// One warp per key: blk_hist[k][b] becomes the number of entries of key k in blocks before
 // b, key_total[k] their total.
 __global__ void __launch_bounds__(256) label_scan_blocks_kernel(uint32_t *__restrict__ blk_hist, int nblk, int KK,
                                                                  uint32_t *__restrict__ key_total)
@@ -75,14 +77,14 @@ __global__ void __launch_bounds__(256) label_scan_blocks_kernel(uint32_t *__rest
     uint32_t carry = 0;
     for (int b0 = 0; b0 < nblk; b0 += 32) {
         const int b = b0 + lane;
-        const uint32_t v = (b < nblk) ? blk_hist[(size_t)b * KK + k] : 0u;
+        const uint32_t v = (b < nblk) ? blk_hist[(size_t)k * nblk + b] : 0u;
         uint32_t incl = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += t;
         }
-        if (b < nblk) blk_hist[(size_t)b * KK + k] = carry + incl - v;
+        if (b < nblk) blk_hist[(size_t)k * nblk + b] = carry + incl - v;
         carry += __shfl_sync(0xffffffffu, incl, 31);
     }
     if (lane == 0) key_total[k] = carry;
@@ -165,7 +167,7 @@ __global__ void __launch_bounds__(SORT_BLOCK) label_scatter_kernel(const int32_t
     }
     __syncthreads();
     if (l >= 0) {
-        const uint32_t pos = (uint32_t)cluster_start[l] + blk_hist[(size_t)blockIdx.x * KK + l] +
+        const uint32_t pos = (uint32_t)cluster_start[l] + blk_hist[(size_t)l * gridDim.x + blockIdx.x] +
                              warp_hist[w * KK + l] + (uint32_t)rank_in_warp;
         order[pos] = (int32_t)(e < N ? e : e - N);
     }
@@ -202,9 +204,8 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
 {
     __shared__ int32_t rows_s[128];
     __shared__ double red_s[SEG_THREADS * VEC];
-    const int seg = blockIdx.x;
     const int nseg_total = p.seg_start[p.K];
-    if (seg >= nseg_total) return;
+    for (int seg = blockIdx.x; seg < nseg_total; seg += gridDim.x) {
     // cluster of this segment: last k with seg_start[k] <= seg
     int lo = 0, hi = p.K;
     while (hi - lo > 1) {
@@ -325,6 +326,8 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
             }
         }
     }
+    __syncthreads();   // red_s and rows_s are reused by the next segment
+    }
 }
 
 // out0/out1[k*D+j] = sum over the segments of key k of plane 0/1 (out1 may be NULL); in
@@ -355,6 +358,53 @@ __global__ void segment_combine_kernel(const double *__restrict__ part, const in
     if (C) {
         const int64_t n = counts[k];
         if (n > 0) C[e] = (float)(a / (double)n);
+    }
+}
+
+// Delta-mode centroid update, one CTA per cluster: S_k += (partials of key k) - (partials of key
+// K + k); c_k = float(S_k / n_k) where n_k > 0; and for the next assignment the squared norm
+// of c_k (fp64, rounded up), optionally the fp16 copy fp16(c_k * scale[0]), and the reset of the
+// exact-pass queues.
+__global__ void __launch_bounds__(256) centroid_update_kernel(const double *__restrict__ part,
+                                                              const int32_t *__restrict__ seg_start,
+                                                              const int64_t *__restrict__ counts, int D, int K,
+                                                              double *__restrict__ sums, float *__restrict__ C,
+                                                              float *__restrict__ cnorm, const float *__restrict__ scale,
+                                                              __half *__restrict__ Ch, Control *ctl)
+{
+    __shared__ double red[8];
+    const int k = blockIdx.x;
+    if (k == 0 && threadIdx.x == 0) {
+        ctl->refine_count = 0;
+        ctl->cand_count = 0;
+    }
+    const int a0 = seg_start[k], a1 = seg_start[k + 1], m0 = seg_start[K + k], m1 = seg_start[K + k + 1];
+    const int64_t n = counts[k];
+    const float sc = Ch ? scale[0] : 1.f;
+    double nrm = 0.0;
+    for (int j = threadIdx.x; j < D; j += blockDim.x) {
+        const size_t e = (size_t)k * D + j;
+        double a = 0.0, m = 0.0;
+        for (int sgm = a0; sgm < a1; ++sgm) a += part[((size_t)sgm * 2) * D + j];
+        for (int sgm = m0; sgm < m1; ++sgm) m += part[((size_t)sgm * 2) * D + j];
+        const double sum = sums[e] + (a - m);
+        sums[e] = sum;
+        float c = C[e];
+        if (n > 0) {
+            c = (float)(sum / (double)n);
+            C[e] = c;
+        }
+        nrm += (double)c * (double)c;
+        if (Ch) Ch[e] = __float2half_rn(c * sc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = nrm;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        cnorm[k] = __double2float_ru(t);
     }
 }
 
@@ -406,7 +456,10 @@ static cudaError_t launch_segment_sums_mode(const SegParams &p, const SegGeom &g
 {
     const bool vec = (p.D % 4 == 0);
     const int units = vec ? p.D / 4 : p.D;
-    dim3 grid((unsigned)g.max_segs, (unsigned)((units + SEG_THREADS - 1) / SEG_THREADS));
+    // a CTA walks segments blockIdx.x, blockIdx.x + gridDim.x, ...: in delta mode most of the
+    // max_segs slots are empty, so the grid stays at a few CTAs per SM
+    const unsigned gx = (unsigned)(g.max_segs < 1184 ? g.max_segs : 1184);
+    dim3 grid(gx, (unsigned)((units + SEG_THREADS - 1) / SEG_THREADS));
     if (vec)
         segment_sums_kernel<MODE, 4><<<grid, SEG_THREADS, 0, s>>>(p);
     else
@@ -448,6 +501,16 @@ cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start,
     const int threads = 256;
     const unsigned blocks = (unsigned)((KD + threads - 1) / threads);
     segment_combine_kernel<<<blocks, threads, 0, s>>>(part, seg_start, counts, D, K, KD, delta ? 1 : 0, out0, out1, C);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_centroid_update(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
+                                   int K, double *sums, float *C, float *cnorm, const float *scale, void *Ch,
+                                   Control *ctl, cudaStream_t s)
+{
+    centroid_update_kernel<<<K, 256, 0, s>>>(part, seg_start, counts, D, K, sums, C, cnorm, scale,
+                                             reinterpret_cast<__half *>(Ch), ctl);
     count_launch();
     return cudaGetLastError();
 }

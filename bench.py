@@ -7,7 +7,7 @@ gamma/beta solve) + cat_apply over one synthetic workload.
 Prints ONE JSON line (rank 0).  `value` is rows through the hot path per second:
 (fit rows x (iters + 1) assignment passes + apply rows) / step time, summed over
 ranks; `apply_rows_per_s` and `fit_s_per_lloyd_iter` give the two quantities
-separately.  Inputs are resident in HBM before the timed region; `e2e` repeats the
+separately (a Lloyd iteration = (fit time - time of the same fit with 0 rounds) / rounds).  Inputs are resident in HBM before the timed region; `e2e` repeats the
 step through the host-buffer entry points with the copies inside the timed region.
 With --impl reference the CPU oracle is timed on a bounded sample of the same
 workload (rank 0 only).
@@ -31,6 +31,10 @@ import numpy as np
 import torch
 
 from paper_2509_26277_b200 import workloads as W
+
+# dram__bytes_read.sum + dram__bytes_write.sum of assign_tc_kernel<affine> per row at D = 1024, K = 256
+# (None while no capture of the current kernel exists)
+APPLY_DRAM_BYTES_PER_ROW = None
 
 METRIC = "CAT rows/s through the hot path (fit row-passes + apply rows); see apply_rows_per_s, fit_s_per_lloyd_iter"
 UNIT = "rows/s"
@@ -246,6 +250,19 @@ def run_cuda(args):
     barrier()
     t_wall = time.perf_counter() - t_wall0
     launches = B.cat_kernel_launches() - launches0
+    # the part of cat_fit that is not a Lloyd round (fp16 copy, final assignment, moments, solve),
+    # timed on its own so that the per-round figure can be separated from it
+    fit0_ms = None
+    if world == 1 and iters > 0:
+        e0 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        B.cat_fit_into(Yq_fit, Yfp_fit, K, 0, C, G, Bt, labels, ws_fit)
+        e0[0].record(stream)
+        for _ in range(args.steps):
+            B.cat_fit_into(Yq_fit, Yfp_fit, K, 0, C, G, Bt, labels, ws_fit)
+        e0[1].record(stream)
+        torch.cuda.synchronize()
+        fit0_ms = e0[0].elapsed_time(e0[1]) / args.steps
+        B.cat_fit_into(Yq_fit, Yfp_fit, K, iters, C, G, Bt, labels, ws_fit)   # leave the fitted model in place
     rep_fit = B.cat_workspace_report(ws_fit) if world == 1 else None
     rep_apply = B.cat_workspace_report(ws_apply)
     clocks = sampler.stop() if rank == 0 else None
@@ -267,9 +284,15 @@ def run_cuda(args):
 
     # dominant kernel: the fused assign+affine kernel of cat_apply (one launch per step).
     # algorithmic bytes per launch = read N*D fp32 + write N*D fp32.
+    # DRAM counter traffic of that kernel (ncu capture at 262 144 rows of this recipe, scaled by
+    # the rows: see profiles/): only meaningful for the shape it was taken on.
+    traffic = APPLY_DRAM_BYTES_PER_ROW * N_apply if (args.config == 4 and APPLY_DRAM_BYTES_PER_ROW) else None
     apply_bytes = 2.0 * N_apply * D * 4
     apply_gbs = apply_bytes / (apply_ms_step * 1e-3) / 1e9
-    lloyd_ms = fit_ms_step / (iters + 1) if iters >= 0 else float("nan")
+    if fit0_ms is not None:
+        lloyd_ms = max(fit_ms_step - fit0_ms, 0.0) / iters
+    else:
+        lloyd_ms = fit_ms_step / (iters + 1)
     lloyd_bytes = 1.0 * N_fit * D * 4
     lloyd_gbs = lloyd_bytes / (lloyd_ms * 1e-3) / 1e9
 
@@ -297,11 +320,11 @@ def run_cuda(args):
                        "parallelism": f"rows x{world}"},
             "apply_rows_per_s": N_apply * world / (apply_ms_step * 1e-3),
             "fit_s_per_lloyd_iter": lloyd_ms * 1e-3,
-            "fit_ms": fit_ms_step, "apply_ms": apply_ms_step,
+            "fit_ms": fit_ms_step, "fit_without_rounds_ms": fit0_ms, "apply_ms": apply_ms_step,
             "wall_s": t_wall,
             "roofline": {"bound": "hbm", "kernel": "assign_tc_kernel<affine, pair> (the one kernel of cat_apply besides the exact pass)",
                          "achieved": apply_gbs, "peak": peak, "unit": "GB/s", "frac": apply_gbs / peak,
-                         "peak_source": peak_src, "traffic": None},
+                         "peak_source": peak_src, "traffic": traffic},
             "roofline_fit": {"bound": "hbm", "kernel": "one Lloyd round of cat_fit (assign_tc_kernel<labels, pair> + exact pass + delta centroid update)",
                              "achieved": lloyd_gbs, "peak": peak, "unit": "GB/s", "frac": lloyd_gbs / peak},
             "exact_pass_rows": {"apply": rep_apply["refined_rows_last"],

@@ -505,12 +505,68 @@ __device__ __forceinline__ void stream_row(const TcParams &p, int64_t row, float
     }
 }
 
+// The same for short rows (D < 128): a row takes only G = 1 .. 16 lanes, so a warp streams all
+// of its rows of the tile (ew, ew + TC_STREAM_WARPS, ...) in one step, 32 / G rows per load slot.
+__device__ __forceinline__ void stream_rows_short(const TcParams &p, int64_t row0, const float4 *tile_keys, int ew,
+                                                  float cmax2, int lane)
+{
+    const int D4 = p.D >> 2;
+    int G = 1;
+    while (G < D4) G <<= 1;
+    const int rps = 32 / G;            // rows per slot
+    const int c = lane & (G - 1);      // float4 column of this lane
+    const int sub = lane / G;          // which of the slot's rows
+    // batches of four load slots (4 * rps rows) until the warp's rows of the tile are done
+#pragma unroll 1
+    for (int i0 = 0; ew + TC_STREAM_WARPS * i0 < TC_BM; i0 += 4 * rps) {
+        float4 y[4], g[4], bb[4];
+        unsigned act = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int r = ew + TC_STREAM_WARPS * (i0 + q * rps + sub);
+            const int64_t row = row0 + r;
+            if ((r < TC_BM) && (row < p.N) && (c < D4)) {
+                act |= 1u << q;
+                const int l = key_label(tile_keys[r].x, p.K);
+                y[q] = __ldcs(reinterpret_cast<const float4 *>(p.Y) + (size_t)row * D4 + c);
+                g[q] = __ldg(reinterpret_cast<const float4 *>(p.gamma) + (size_t)l * D4 + c);
+                bb[q] = __ldg(reinterpret_cast<const float4 *>(p.beta) + (size_t)l * D4 + c);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float ysq = 0.f;
+            const int r = ew + TC_STREAM_WARPS * (i0 + q * rps + sub);
+            const int64_t row = row0 + r;
+            if (act & (1u << q)) {
+                float4 v;
+                v.x = fmaf(g[q].x, y[q].x, bb[q].x);
+                v.y = fmaf(g[q].y, y[q].y, bb[q].y);
+                v.z = fmaf(g[q].z, y[q].z, bb[q].z);
+                v.w = fmaf(g[q].w, y[q].w, bb[q].w);
+                __stcs(reinterpret_cast<float4 *>(p.out) + (size_t)row * D4 + c, v);
+                ysq = fmaf(y[q].x, y[q].x, fmaf(y[q].y, y[q].y, fmaf(y[q].z, y[q].z, y[q].w * y[q].w)));
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1)
+                if (o < G) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
+            if ((act & (1u << q)) && c == 0) {
+                const float4 keys = tile_keys[r];
+                const float e = tc_error_bound(p.D, ysq * 1.0001f, cmax2);
+                p.labels[row] = key_label(keys.x, p.K);
+                tc_decide(p, row, keys, e);
+            }
+        }
+    }
+}
+
 // PAIR: the two CTAs of a cluster work as one cta_group::2 unit on 256 rows.  Each CTA
 // loads the slabs of its own 128 rows and of HALF the centroids; the MMA (M = 256, issued
 // by the CTA of rank 0) reads both halves, and each CTA finds the scores of its own rows in
 // its own TMEM.
 // HALF: operands are the fp16 copies of the rows and centroids (64 columns per slab, kind::f16).
-template <bool AFFINE, bool PAIR, bool HALF>
+// SHORT (affine epilogue only): rows of fewer than 128 columns, streamed several per warp step.
+template <bool AFFINE, bool PAIR, bool HALF, bool SHORT>
 __global__ void __launch_bounds__(AFFINE ? TC_THREADS_AFFINE : TC_THREADS_LABELS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p)
 {
@@ -772,11 +828,17 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
             if (!mbar_wait_warp(smem_u32(&sh.lab_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
             if (ew == 0 && lane == 0) TC_TRACE(ti, 6);
-            for (int r = ew; r < TC_BM; r += TC_STREAM_WARPS) {
-                const int64_t row = row0 + r;
-                if (row < p.N) stream_row(p, row, sh.top_key[b][r], cmax2, lane);
+            if (SHORT) {
+                stream_rows_short(p, row0, sh.top_key[b], ew, cmax2, lane);
                 __syncwarp();
-                if (lane == 0) atomicAdd(&sh.rows_streamed, 1);
+                if (lane == 0) atomicAdd(&sh.rows_streamed, (TC_BM - ew + TC_STREAM_WARPS - 1) / TC_STREAM_WARPS);
+            } else {
+                for (int r = ew; r < TC_BM; r += TC_STREAM_WARPS) {
+                    const int64_t row = row0 + r;
+                    if (row < p.N) stream_row(p, row, sh.top_key[b][r], cmax2, lane);
+                    __syncwarp();
+                    if (lane == 0) atomicAdd(&sh.rows_streamed, 1);
+                }
             }
             __syncwarp();
             if (ew == 0 && lane == 0) TC_TRACE(ti, 7);
@@ -796,53 +858,38 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     }
 }
 
-// squared row norms (labels-only mode): one warp per row
-__global__ void row_norms_kernel(const float *__restrict__ Y, int64_t N, int D, float *__restrict__ out)
+// Squared row norms (labels-only mode), slightly over-estimated to keep the error bound on the safe
+// side; with amax_bits also the largest magnitude of the matrix (as the bits of a non-negative float,
+// which order like unsigned integers).  A row is read by G lanes, G = the power of two >= D / 4
+// capped at 32, so short rows share a warp.
+__global__ void row_norms_kernel(const float *__restrict__ Y, int64_t N, int D, int G, float *__restrict__ out,
+                                 unsigned int *__restrict__ amax_bits)
 {
-    const int lane = threadIdx.x & 31;
-    const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (row >= N) return;
-    const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)row * D);
-    float s = 0.f;
-    for (int c = lane; c < (D >> 2); c += 32) {
-        float4 v = __ldg(y4 + c);
-        s = fmaf(v.x, v.x, s);
-        s = fmaf(v.y, v.y, s);
-        s = fmaf(v.z, v.z, s);
-        s = fmaf(v.w, v.w, s);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    // a slight over-estimate keeps the error bound on the safe side
-    if (lane == 0) out[row] = s * 1.0001f;
-}
-
-// Squared row norms as above, and the largest magnitude of the matrix (as the bits of a
-// non-negative float, which order like unsigned integers) into scale_bits[0].
-__global__ void row_norms_amax_kernel(const float *__restrict__ Y, int64_t N, int D, float *__restrict__ out,
-                                      unsigned int *__restrict__ amax_bits)
-{
-    const int lane = threadIdx.x & 31;
-    const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (row >= N) return;
-    const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)row * D);
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t row = t / G;
+    const int c0 = (int)(t % G);
     float s = 0.f, m = 0.f;
-    for (int c = lane; c < (D >> 2); c += 32) {
-        float4 v = __ldg(y4 + c);
-        s = fmaf(v.x, v.x, s);
-        s = fmaf(v.y, v.y, s);
-        s = fmaf(v.z, v.z, s);
-        s = fmaf(v.w, v.w, s);
-        m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+    if (row < N) {
+        const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)row * D);
+        for (int c = c0; c < (D >> 2); c += G) {
+            float4 v = __ldg(y4 + c);
+            s = fmaf(v.x, v.x, s);
+            s = fmaf(v.y, v.y, s);
+            s = fmaf(v.z, v.z, s);
+            s = fmaf(v.w, v.w, s);
+            m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        s += __shfl_xor_sync(0xffffffffu, s, o);
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (o < G) {
+            s += __shfl_xor_sync(0xffffffffu, s, o);
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        }
     }
-    if (lane == 0) {
+    if (row < N && c0 == 0) {
         out[row] = s * 1.0001f;
-        if (m == m && m < CUDART_INF_F) atomicMax(amax_bits, __float_as_uint(m));
+        if (amax_bits && m == m && m < CUDART_INF_F) atomicMax(amax_bits, __float_as_uint(m));
     }
 }
 
@@ -928,6 +975,13 @@ bool regs_ok(const void *kern)
     return (long)a.numRegs * TC_THREADS_AFFINE >= 128L * (TC_REGS_CONTROL + TC_REGS_SCORE + 3 * TC_REGS_STREAM);
 }
 
+int lanes_per_row(int D)
+{
+    int G = 1;
+    while (G < (D >> 2) && G < 32) G <<= 1;
+    return G;
+}
+
 int sm_count()
 {
     static int cached[64] = {};
@@ -951,8 +1005,9 @@ bool tc_supported(int64_t N, int D, int K)
 cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaStream_t s)
 {
     const int threads = 256;
-    const int64_t blocks = (N * 32 + threads - 1) / threads;
-    row_norms_kernel<<<(unsigned)blocks, threads, 0, s>>>(Y, N, D, out);
+    const int G = lanes_per_row(D);
+    const int64_t blocks = (N * G + threads - 1) / threads;
+    row_norms_kernel<<<(unsigned)blocks, threads, 0, s>>>(Y, N, D, G, out, nullptr);
     count_launch();
     return cudaGetLastError();
 }
@@ -963,8 +1018,9 @@ cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, 
     cudaError_t e = cudaMemsetAsync(scale, 0, 4 * sizeof(float), s);
     if (e != cudaSuccess) return e;
     const int threads = 256;
-    const int64_t blocks = (N * 32 + threads - 1) / threads;
-    row_norms_amax_kernel<<<(unsigned)blocks, threads, 0, s>>>(Y, N, D, ynorm2, reinterpret_cast<unsigned int *>(scale));
+    const int G = lanes_per_row(D);
+    const int64_t blocks = (N * G + threads - 1) / threads;
+    row_norms_kernel<<<(unsigned)blocks, threads, 0, s>>>(Y, N, D, G, ynorm2, reinterpret_cast<unsigned int *>(scale));
     half_scale_kernel<<<1, 32, 0, s>>>(scale);
     const size_t n4 = (size_t)N * D / 4;
     size_t cb = (n4 + threads - 1) / threads;
@@ -1070,9 +1126,9 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     cfg.numAttrs = 1;
 
     cudaError_t e;
-#define CAT_TC_LAUNCH(AFF, PR, HF)                                                                                      \
+#define CAT_TC_LAUNCH(AFF, PR, HF, SH)                                                                                      \
     do {                                                                                                               \
-        auto kern = assign_tc_kernel<AFF, PR, HF>;                                                                      \
+        auto kern = assign_tc_kernel<AFF, PR, HF, SH>;                                                                      \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)   \
             return e;                                                                                                  \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, carveout)) != cudaSuccess) \
@@ -1080,12 +1136,14 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
         if (AFF && !regs_ok(reinterpret_cast<const void *>(kern))) return cudaErrorLaunchOutOfResources;               \
         e = cudaLaunchKernelEx(&cfg, kern, mapA, mapB, p);                                                             \
     } while (0)
-    if (affine) {
-        if (pair) CAT_TC_LAUNCH(true, true, false); else CAT_TC_LAUNCH(true, false, false);
+    if (affine && D < 128) {
+        if (pair) CAT_TC_LAUNCH(true, true, false, true); else CAT_TC_LAUNCH(true, false, false, true);
+    } else if (affine) {
+        if (pair) CAT_TC_LAUNCH(true, true, false, false); else CAT_TC_LAUNCH(true, false, false, false);
     } else if (half) {
-        if (pair) CAT_TC_LAUNCH(false, true, true); else CAT_TC_LAUNCH(false, false, true);
+        if (pair) CAT_TC_LAUNCH(false, true, true, false); else CAT_TC_LAUNCH(false, false, true, false);
     } else {
-        if (pair) CAT_TC_LAUNCH(false, true, false); else CAT_TC_LAUNCH(false, false, false);
+        if (pair) CAT_TC_LAUNCH(false, true, false, false); else CAT_TC_LAUNCH(false, false, false, false);
     }
 #undef CAT_TC_LAUNCH
     if (e != cudaSuccess) return e;

@@ -169,6 +169,47 @@ def test_ragged_shapes_apply_and_fit(n, d, k):
             assert np.array_equal(host(lg), ora.labels)
 
 
+@pytest.mark.parametrize("n,d,k,scale", [(600, 2048, 40, 1.0),      # rows longer than one streaming step
+                                         (300, 120, 33, 1.0),       # short rows, 30 float4 (not a power of two)
+                                         (700, 1032, 64, 1.0),      # last fp16 slab partly outside the matrix
+                                         (520, 1028, 48, 1.0),      # D % 8 != 0: the fit stays on TF32 operands
+                                         (3000, 256, 128, 1.0),
+                                         (1500, 512, 256, 3.0e4),   # magnitudes far above the fp16 range
+                                         (1500, 512, 256, 2.0e-7)])  # ... and far below it
+def test_tensor_paths_shapes_and_scales(n, d, k, scale):
+    """Shapes and magnitudes that steer the tensor-core kernels through their variants (fp16 copy of
+    the rows with its power-of-two scale, TF32, short and long rows).  Tolerances scale with the data."""
+    Yq = (_rand(n + d, n, d) * scale).astype(np.float32)
+    Yfp = (Yq * 0.9 + 0.05 * scale * _rand(n + d + 1, n, d)).astype(np.float32)
+    Cg, Gg, Bg, lg = B.cat_fit(dev(Yq), dev(Yfp), k, 4)
+    lab, best, second = O.assign(Yq, host(Cg))
+    labels_match(host(lg), lab, best, second, "fit labels")
+    g_want, b_want = O.solve_gamma_beta(Yq, Yfp, host(lg), k)
+    close(host(Gg), g_want, "gamma")
+    close(host(Bg) / scale, b_want / scale, "beta")
+    ora = O.fit(Yq, Yfp, k, 4, near_rel=1e-5)
+    if ora.near.sum() == 0:
+        assert np.array_equal(host(lg), ora.labels)
+        close(host(Cg) / scale, ora.centroids / scale, "centroids")
+    want, lab, best, second = O.apply(Yq, host(Cg), host(Gg), host(Bg))
+    out, glab = B.cat_apply(dev(Yq), Cg, Gg, Bg, want_labels=True)
+    _, n_diff = labels_match(host(glab), lab, best, second, "apply labels")
+    want2 = want if n_diff == 0 else O.affine_with_labels(Yq, host(glab), host(Gg), host(Bg))
+    close(host(out) / scale, want2 / scale, "outputs")
+
+
+def test_fit_fp16_and_tf32_operands_agree():
+    """The default start lets cat_fit assign from an fp16 copy of the rows; an explicit start (here the
+    same first K rows) keeps TF32 operands.  Labels are decided exactly either way."""
+    w, _ = workload("cfg4s")
+    Yq, Yfp = dev(w.Yq_fit.numpy()), dev(w.Yfp_fit.numpy())
+    a = B.cat_fit(Yq, Yfp, w.K, 6)
+    b = B.cat_fit(Yq, Yfp, w.K, 6, init_centroids=Yq[:w.K].clone())
+    assert torch.equal(a[3], b[3])
+    for x, y in zip(a[:3], b[:3]):
+        close(host(x), host(y), "fp16 vs tf32 fit")
+
+
 def test_exact_ties_resolve_to_lowest_index():
     Yq = np.array([[0, 0, 0, 0], [1, 0, 0, 0], [5, 5, 5, 5]] * 50, np.float32)
     C = np.array([[-1, 0, 0, 0], [5, 5, 5, 5], [1, 0, 0, 0], [5, 5, 5, 5]], np.float32)

@@ -62,7 +62,12 @@ FitWs carve_fit(void *base, int64_t N, int D, int K)
     w.seg_start = c.take<int32_t>((size_t)2 * K + 1);
     w.order = c.take<int32_t>((size_t)2 * N);
     w.labels_prev = c.take<int32_t>((size_t)N);
-    w.segpart = c.take<double>((size_t)g.max_segs * 2 * D);
+    {
+        // two planes per segment in delta mode, three in the single-sweep final pass (full mode)
+        const SegGeom gf = seg_geometry(N, D, K);
+        const size_t a = (size_t)g.max_segs * 2, b = (size_t)gf.max_segs * 3;
+        w.segpart = c.take<double>((a > b ? a : b) * D);
+    }
     w.yh = c.take<uint16_t>((size_t)N * D);
     w.ch = c.take<uint16_t>(KD);
     w.hscale = c.take<float>(4);
@@ -259,7 +264,7 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     FitWs w = carve_fit(workspace, N, D, K);
     const size_t KD = (size_t)K * D;
-    double *meanQ = w.meanQ, *meanF = w.meanF;
+    double *meanQ = w.meanQ;
     int32_t *labels = labels_out ? labels_out : w.a.labels;
     float *C = centroids_out;
 
@@ -297,18 +302,26 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale,
                     iters > 0);
     if (st != CAT_OK) return st;
+    // The running sums follow the final labels too (without touching the centroids), which gives
+    // the cluster means of Yq before the one sweep over Yq and Yfp that forms the centred moments
+    // and the sums of Yfp.
+    {
+        SegGeom gd = seg_geometry(2 * N, D, 2 * K);
+        CAT_CUDA(launch_label_sort(labels, lab[1], N, K, gd, w.blk_hist, w.key_total, w.counts, w.cluster_start,
+                                   w.seg_start, w.order, s));
+        CAT_CUDA(launch_segment_sums(0, Yq, nullptr, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D,
+                                     2 * K, gd, w.segpart, s));
+        CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, true, w.sumQ, nullptr, nullptr, s));
+    }
+    CAT_CUDA(launch_means_from_sums(w.sumQ, w.counts, D, K, meanQ, s));
     st = run_sort(labels, N, D, K, w, w.counts, s);
     if (st != CAT_OK) return st;
     {
         SegGeom g = seg_geometry(N, D, K);
-        CAT_CUDA(launch_segment_sums(1, Yq, Yfp, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D,
-                                     K, g, w.segpart, s));
-        CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, false, w.sumQ, w.sumF, nullptr, s));
+        CAT_CUDA(launch_segment_sums(3, Yq, Yfp, w.order, w.cluster_start, w.seg_start, meanQ, nullptr, D, K, g,
+                                     w.segpart, s));
+        CAT_CUDA(launch_segment_combine3(w.segpart, w.seg_start, D, K, w.var, w.cov, w.sumF, s));
     }
-    CAT_CUDA(launch_means_from_sums(w.sumQ, w.counts, D, K, meanQ, s));
-    CAT_CUDA(launch_means_from_sums(w.sumF, w.counts, D, K, meanF, s));
-    st = run_centred(Yq, Yfp, N, D, K, w, meanQ, meanF, w.var, w.cov, s);
-    if (st != CAT_OK) return st;
     CAT_CUDA(launch_solve(w.sumQ, w.sumF, w.var, w.cov, w.counts, D, K, gamma_out, beta_out, s));
     if (diag) CAT_CUDA(launch_fit_diag(w.a.ctl, w.counts, K, diag, s));
     return CAT_OK;

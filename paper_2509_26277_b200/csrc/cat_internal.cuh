@@ -132,7 +132,8 @@ cudaError_t launch_label_sort(const int32_t *labels, const int32_t *prev, int64_
 
 // Per-segment partial sums over KK keys.  mode 0: column sums of Yq (plane 0); mode 1: of Yq and Yf
 // (planes 0, 1); mode 2 (full mode only): centred moments sum (q-muQ)^2 (plane 0) and
-// sum (q-muQ)(f-muF) (plane 1).
+// sum (q-muQ)(f-muF) (plane 1); mode 3 (full mode only, three planes per segment): sum (q-muQ)^2,
+// sum (q-muQ)(f-muQ), sum f.
 cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, const int32_t *order,
                                 const int32_t *cluster_start, const int32_t *seg_start, const double *meanQ,
                                 const double *meanF, int D, int KK, const SegGeom &g, double *part,
@@ -143,6 +144,10 @@ cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, cons
 // float(out0 / n_k) for clusters with n_k > 0.
 cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start, const int64_t *counts, int D,
                                    int K, bool delta, double *out0, double *out1, float *C, cudaStream_t s);
+
+// Sums of the three planes of mode 3 per cluster: out0 = sum (q-muQ)^2, out1 = sum (q-muQ)(f-muQ), out2 = sum f.
+cudaError_t launch_segment_combine3(const double *part, const int32_t *seg_start, int D, int K, double *out0,
+                                    double *out1, double *out2, cudaStream_t s);
 
 // Delta-mode centroid update fused with what the next assignment needs: running sums, centroids,
 // their squared norms, (with Ch) their fp16 copy, and the reset of the exact-pass queues.

@@ -196,8 +196,36 @@ __device__ __forceinline__ void add4(double (&a)[4], const float4 v)
     a[3] += (double)v.w;
 }
 
+// One row's contribution (VEC columns) to the accumulators of a segment.
+template <int MODE, int VEC>
+__device__ __forceinline__ void seg_accumulate(double (&a0)[4], double (&a1)[4], double (&a2)[4], const double (&mq)[4],
+                                               const double (&mf)[4], const float4 q4, const float4 f4)
+{
+    if (MODE == 0) {
+        add4(a0, q4);
+    } else if (MODE == 1) {
+        add4(a0, q4);
+        add4(a1, f4);
+    } else {
+        const float qv[4] = {q4.x, q4.y, q4.z, q4.w};
+        const float fv[4] = {f4.x, f4.y, f4.z, f4.w};
+#pragma unroll
+        for (int q = 0; q < VEC; ++q) {
+            const double dq = (double)qv[q] - mq[q];
+            const double df = (double)fv[q] - mf[q];
+            a0[q] = fma(dq, dq, a0[q]);
+            a1[q] = fma(dq, df, a1[q]);
+            if (MODE == 3) a2[q] += (double)fv[q];
+        }
+    }
+}
+
 // MODE 0: sums of Yq -> plane 0.  MODE 1: sums of Yq, Yf -> planes 0, 1.
 // MODE 2: centred moments -> plane 0 = sum (q-muQ)^2, plane 1 = sum (q-muQ)(f-muF).
+// MODE 3: the final pass of cat_fit in one sweep, with the cluster mean muQ known beforehand:
+//         plane 0 = sum (q-muQ)^2, plane 1 = sum (q-muQ)(f-muQ), plane 2 = sum f (three planes
+//         per segment).  Since sum (q-muQ) = 0, plane 1 is the centred cross moment whatever
+//         constant is subtracted from f; muQ keeps the products small.
 // VEC: 4 = 128-bit loads (D % 4 == 0), 1 = scalar loads.
 template <int MODE, int VEC>
 __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
@@ -228,13 +256,13 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
     const bool active = (c < SEG_THREADS) && (unit < units);
     const int col = unit * VEC;
 
-    double a0[4] = {0, 0, 0, 0}, a1[4] = {0, 0, 0, 0};
+    double a0[4] = {0, 0, 0, 0}, a1[4] = {0, 0, 0, 0}, a2[4] = {0, 0, 0, 0};
     double mq[4] = {0, 0, 0, 0}, mf[4] = {0, 0, 0, 0};
-    if (MODE == 2 && active) {
+    if (MODE >= 2 && active) {
 #pragma unroll
         for (int q = 0; q < VEC; ++q) {
             mq[q] = p.meanQ[(size_t)k * p.D + col + q];
-            mf[q] = p.meanF[(size_t)k * p.D + col + q];
+            mf[q] = (MODE == 2) ? p.meanF[(size_t)k * p.D + col + q] : mq[q];
         }
     }
 
@@ -260,24 +288,7 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (MODE == 0) {
-                    add4(a0, q4[u]);
-                } else if (MODE == 1) {
-                    add4(a0, q4[u]);
-                    add4(a1, f4[u]);
-                } else {
-                    const float qv[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
-                    const float fv[4] = {f4[u].x, f4[u].y, f4[u].z, f4[u].w};
-#pragma unroll
-                    for (int q = 0; q < VEC; ++q) {
-                        const double dq = (double)qv[q] - mq[q];
-                        const double df = (double)fv[q] - mf[q];
-                        a0[q] = fma(dq, dq, a0[q]);
-                        a1[q] = fma(dq, df, a1[q]);
-                    }
-                }
-            }
+            for (int u = 0; u < 4; ++u) seg_accumulate<MODE, VEC>(a0, a1, a2, mq, mf, q4[u], f4[u]);
         }
         for (; r < nb; r += G) {
             const size_t o = (size_t)rows_s[r] * p.D + col;
@@ -289,35 +300,21 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
                 q4 = make_float4(__ldg(p.Yq + o), 0.f, 0.f, 0.f);
                 if (MODE != 0) f4 = make_float4(__ldg(p.Yf + o), 0.f, 0.f, 0.f);
             }
-            if (MODE == 0) {
-                add4(a0, q4);
-            } else if (MODE == 1) {
-                add4(a0, q4);
-                add4(a1, f4);
-            } else {
-                const float qv[4] = {q4.x, q4.y, q4.z, q4.w};
-                const float fv[4] = {f4.x, f4.y, f4.z, f4.w};
-#pragma unroll
-                for (int q = 0; q < VEC; ++q) {
-                    const double dq = (double)qv[q] - mq[q];
-                    const double df = (double)fv[q] - mf[q];
-                    a0[q] = fma(dq, dq, a0[q]);
-                    a1[q] = fma(dq, df, a1[q]);
-                }
-            }
+            seg_accumulate<MODE, VEC>(a0, a1, a2, mq, mf, q4, f4);
         }
     }
 
     // add the row groups in a fixed order and publish the segment's partial row
-    constexpr int NPLANES = (MODE == 0) ? 1 : 2;
+    constexpr int NPLANES = (MODE == 0) ? 1 : (MODE == 3 ? 3 : 2);
+    constexpr int PSTRIDE = (MODE == 3) ? 3 : 2;   // planes per segment in `part`
 #pragma unroll
     for (int pl = 0; pl < NPLANES; ++pl) {
         __syncthreads();
 #pragma unroll
-        for (int q = 0; q < VEC; ++q) red_s[tid * VEC + q] = (pl == 0) ? a0[q] : a1[q];
+        for (int q = 0; q < VEC; ++q) red_s[tid * VEC + q] = (pl == 0) ? a0[q] : (pl == 1 ? a1[q] : a2[q]);
         __syncthreads();
         if (g == 0 && active) {
-            double *dst = p.part + ((size_t)seg * 2 + pl) * p.D + col;
+            double *dst = p.part + ((size_t)seg * PSTRIDE + pl) * p.D + col;
 #pragma unroll
             for (int q = 0; q < VEC; ++q) {
                 double s = 0.0;
@@ -359,6 +356,26 @@ __global__ void segment_combine_kernel(const double *__restrict__ part, const in
         const int64_t n = counts[k];
         if (n > 0) C[e] = (float)(a / (double)n);
     }
+}
+
+// Three-plane partials (MODE 3) added up per cluster.
+__global__ void segment_combine3_kernel(const double *__restrict__ part, const int32_t *__restrict__ seg_start, int D,
+                                        size_t KD, double *__restrict__ out0, double *__restrict__ out1,
+                                        double *__restrict__ out2)
+{
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= KD) return;
+    const int k = (int)(e / D);
+    const int j = (int)(e - (size_t)k * D);
+    double a = 0.0, b = 0.0, c = 0.0;
+    for (int sgm = seg_start[k]; sgm < seg_start[k + 1]; ++sgm) {
+        a += part[((size_t)sgm * 3) * D + j];
+        b += part[((size_t)sgm * 3 + 1) * D + j];
+        c += part[((size_t)sgm * 3 + 2) * D + j];
+    }
+    out0[e] = a;
+    out1[e] = b;
+    out2[e] = c;
 }
 
 // Delta-mode centroid update, one CTA per cluster: S_k += (partials of key k) - (partials of key
@@ -490,7 +507,8 @@ cudaError_t launch_segment_sums(int mode, const float *Yq, const float *Yf, cons
     switch (mode) {
     case 0: return launch_segment_sums_mode<0>(p, g, s);
     case 1: return launch_segment_sums_mode<1>(p, g, s);
-    default: return launch_segment_sums_mode<2>(p, g, s);
+    case 2: return launch_segment_sums_mode<2>(p, g, s);
+    default: return launch_segment_sums_mode<3>(p, g, s);
     }
 }
 
@@ -501,6 +519,17 @@ cudaError_t launch_segment_combine(const double *part, const int32_t *seg_start,
     const int threads = 256;
     const unsigned blocks = (unsigned)((KD + threads - 1) / threads);
     segment_combine_kernel<<<blocks, threads, 0, s>>>(part, seg_start, counts, D, K, KD, delta ? 1 : 0, out0, out1, C);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_segment_combine3(const double *part, const int32_t *seg_start, int D, int K, double *out0,
+                                    double *out1, double *out2, cudaStream_t s)
+{
+    const size_t KD = (size_t)K * D;
+    const int threads = 256;
+    const unsigned blocks = (unsigned)((KD + threads - 1) / threads);
+    segment_combine3_kernel<<<blocks, threads, 0, s>>>(part, seg_start, D, KD, out0, out1, out2);
     count_launch();
     return cudaGetLastError();
 }

@@ -871,13 +871,22 @@ __global__ void row_norms_kernel(const float *__restrict__ Y, int64_t N, int D, 
     float s = 0.f, m = 0.f;
     if (row < N) {
         const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)row * D);
-        for (int c = c0; c < (D >> 2); c += G) {
-            float4 v = __ldg(y4 + c);
-            s = fmaf(v.x, v.x, s);
-            s = fmaf(v.y, v.y, s);
-            s = fmaf(v.z, v.z, s);
-            s = fmaf(v.w, v.w, s);
-            m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+        const int D4 = D >> 2;
+        for (int c = c0; c < D4; c += 8 * G) {   // eight loads in flight per lane
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int cc = c + u * G;
+                v[u] = (cc < D4) ? __ldg(y4 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                s = fmaf(v[u].x, v[u].x, s);
+                s = fmaf(v[u].y, v[u].y, s);
+                s = fmaf(v[u].z, v[u].z, s);
+                s = fmaf(v[u].w, v[u].w, s);
+                m = fmaxf(fmaxf(m, fmaxf(fabsf(v[u].x), fabsf(v[u].y))), fmaxf(fabsf(v[u].z), fabsf(v[u].w)));
+            }
         }
     }
 #pragma unroll

@@ -70,7 +70,7 @@ FitWs carve_fit(void *base, int64_t N, int D, int K)
     }
     w.yh = c.take<uint16_t>((size_t)N * D);
     w.ch = c.take<uint16_t>(KD);
-    w.hscale = c.take<float>(4);
+    w.hscale = c.take<float>(4 + (size_t)N);
     w.sumQ = c.take<double>(KD);
     w.sumF = c.take<double>(KD);
     w.var = c.take<double>(KD);

@@ -72,7 +72,7 @@ struct FitWs {
     double *segpart;       // [max_segs][2][D] per-segment partial sums
     void *yh;              // [N*D] fp16 copy of Yq (tensor-core fits with D % 8 == 0)
     void *ch;              // [K*D] fp16 copy of the centroids
-    float *hscale;         // [4] scale of the fp16 copies
+    float *hscale;         // [4 + N] scale of the fp16 centroids, then the inverse row scales
     double *sumQ, *sumF, *var, *cov;   // [K*D] each
     double *meanQ, *meanF;             // [K*D] each
     int64_t *counts;       // [K]
@@ -108,8 +108,9 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
                              const float *gamma, const float *beta, float *out, cudaStream_t s,
                              const void *Yh = nullptr, const void *Ch = nullptr, const float *scale = nullptr);
 
-// fp16 copy of a matrix for repeated assignments: squared row norms, scale[4] (power-of-two scale,
-// -2 / scale^2, subnormal rounding error) and Yh = fp16(Y * scale).  Needs D % 8 == 0.
+// fp16 copy of a matrix for repeated assignments, made in one sweep: squared row norms, per-row
+// power-of-two scales, Yh[i] = fp16(Y[i] * scale_i), and scale[4 + N] = {centroid scale s_c from the
+// largest magnitude, -2 / s_c, 2^-25 / s_c, unused, then 1 / scale_i for every row}.  Needs D % 8 == 0.
 bool tc_half_supported(int64_t N, int D, int K);
 cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, float *scale, void *Yh,
                                cudaStream_t s);

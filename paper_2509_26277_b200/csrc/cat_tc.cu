@@ -17,12 +17,14 @@
 // tensor core taken as <= 2^-22 per term; the last term is the index packed into the
 // key).  Rows it cannot decide go to the same exact fp64 pass, so labels stay exact.
 //
-// cat_fit assigns the same rows many times, so it keeps an fp16 copy of them (scaled by a
-// power of two so that the largest magnitude sits near 2^14, rounded to nearest) and runs the
-// labels kernel on that copy with kind::f16: twice the MMA rate of TF32, half the row bytes,
-// and a tighter operand bound (2^-11 per operand instead of 2^-10):
-//     e <= (2^-9 + (2D+2) 2^-22) ||y|| cmax + 2 a sqrt(D) (||y|| + cmax) + 2 D a^2 + 4 u cmax^2 + (packing term)
-// where a = 2^-25 / scale is the absolute rounding error of an element in fp16's subnormal range.
+// cat_fit assigns the same rows many times, so it keeps an fp16 copy of them (each row scaled
+// by its own power of two so that its largest magnitude sits near 2^14, rounded to nearest;
+// the centroids by one power of two taken from the largest magnitude of the whole matrix) and
+// runs the labels kernel on that copy with kind::f16: twice the MMA rate of TF32, half the row
+// bytes, and a tighter operand bound (2^-11 per operand instead of 2^-10):
+//     e <= (2^-9 + (2D+2) 2^-22) ||y|| cmax + 2 sqrt(D) (a_c ||y|| + a_y cmax) + 2 D a_y a_c + 4 u cmax^2 + (packing term)
+// where a_y = 2^-25 / (row scale), a_c = 2^-25 / (centroid scale) are the absolute rounding
+// errors of an element that falls into fp16's subnormal range.
 //
 // For inference, streaming warps then read every row of the tile once more and write
 // gamma_l * y + beta_l for the fast label l; an undecided row is queued and the exact pass
@@ -348,7 +350,8 @@ struct TcParams {
     const float *Y;
     const float *cnorm;
     const float *ynorm2;   // [N] squared row norms (labels-only mode)
-    const float *scale;    // fp16 operands: {scale, -2 / scale^2, 2^-25 / scale} in device memory
+    const float *scale;    // fp16 operands: {centroid scale s_c, -2 / s_c, 2^-25 / s_c, -} followed by
+                           // [N] 1 / (row scale), in device memory
     int32_t *labels;
     int32_t *refine_rows;
     int32_t *cand_rows;    // rows whose exact decision only needs the listed candidates
@@ -419,16 +422,16 @@ __device__ __forceinline__ float tc_error_bound(int D, float ysq, float cmax2)
     return 1.0625f * ((a + 2.f * pk) * yc + (4.f * u + pk) * cmax2);
 }
 
-// Same for fp16 operands (round to nearest, scaled by a power of two; a = absolute rounding
-// error of an element that falls into fp16's subnormal range).
-__device__ __forceinline__ float tc_error_bound_half(int D, float ysq, float cmax2, float a)
+// Same for fp16 operands (round to nearest, scaled by powers of two; ay, ac = absolute rounding
+// error of a row / centroid element that falls into fp16's subnormal range).
+__device__ __forceinline__ float tc_error_bound_half(int D, float ysq, float cmax2, float ay, float ac)
 {
     const float u = 5.9604645e-8f;   // 2^-24
     const float r = 1.953125e-3f * 1.001f + (2.f * (float)D + 2.f) * 2.3841858e-7f;  // 2^-9 (1 + 2^-12) + (2D+2) 2^-22
     const float pk = 3.0517578e-5f;
     const float yn = sqrtf(ysq), cn = sqrtf(cmax2);
-    return 1.0625f * ((r + 2.f * pk) * yn * cn + 2.f * a * sqrtf((float)D) * (yn + cn) + 2.f * (float)D * a * a +
-                      (4.f * u + pk) * cmax2);
+    return 1.0625f * ((r + 2.f * pk) * yn * cn + 2.f * sqrtf((float)D) * (ac * yn + ay * cn) +
+                      2.f * (float)D * ay * ac + (4.f * u + pk) * cmax2);
 }
 
 // Decision for one row from its four smallest keys.  Returns true when the fast argmin is
@@ -590,8 +593,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     const int64_t unit_step = PAIR ? (int64_t)(gridDim.x >> 1) : (int64_t)gridDim.x;
     constexpr int BK = HALF ? 64 : 32;   // columns per slab
     const int nslabs = (p.D + BK - 1) / BK;
-    const float coef = HALF ? p.scale[1] : -2.f;               // score = cn + coef * accumulator
-    const float abs_err = HALF ? p.scale[2] : 0.f;
+    const float coef_c = HALF ? p.scale[1] : -2.f;             // score = cn + coef * accumulator
+    const float abs_err_c = HALF ? p.scale[2] : 0.f;
 
     if (tid == 0) {
         for (int s = 0; s < na; ++s) {
@@ -774,6 +777,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
             tc_fence_after();
             if (quarter == 0 && lane == 0) TC_TRACE(ti, 4);
+            // fp16 operands: this thread's row has its own scale
+            float rinv = 1.f;
+            if (HALF && row0 + quarter * 32 + lane < p.N) rinv = p.scale[4 + row0 + quarter * 32 + lane];
+            const float coef = coef_c * rinv;
             float b1 = TC_KEY_INIT, b2 = TC_KEY_INIT, b3 = TC_KEY_INIT, b4 = TC_KEY_INIT;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
             // two register buffers: the next 16 columns are in flight while these are scanned
@@ -809,7 +816,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             } else {
                 const int64_t row = row0 + r;
                 if (row < p.N) {
-                    const float e = HALF ? tc_error_bound_half(p.D, p.ynorm2[row], cmax2, abs_err)
+                    const float e = HALF ? tc_error_bound_half(p.D, p.ynorm2[row], cmax2, 2.9802322e-8f * rinv, abs_err_c)
                                          : tc_error_bound(p.D, p.ynorm2[row], cmax2);
                     p.labels[row] = key_label(b1, p.K);
                     tc_decide(p, row, make_float4(b1, b2, b3, b4), e);
@@ -902,9 +909,9 @@ __global__ void row_norms_kernel(const float *__restrict__ Y, int64_t N, int D, 
     }
 }
 
-// scale[0] = power of two that brings the largest magnitude to [2^13, 2^14); scale[1] = -2 / scale^2
-// (turns the fp16 accumulator into -2 y.c); scale[2] = 2^-25 / scale (rounding error, in the units
-// of the data, of an element that lands in fp16's subnormal range).
+// scale[0] = s_c, the power of two that brings the largest magnitude of the matrix (the bits
+// left in scale[0] by the shadow kernel) to [2^13, 2^14); scale[1] = -2 / s_c (times 1 / row scale
+// it turns the fp16 accumulator into -2 y.c); scale[2] = 2^-25 / s_c.
 __global__ void half_scale_kernel(float *scale)
 {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
@@ -916,8 +923,80 @@ __global__ void half_scale_kernel(float *scale)
     if (sh < -100) sh = -100;
     const float sc = ldexpf(1.f, sh);
     scale[0] = sc;
-    scale[1] = -2.f / (sc * sc);
+    scale[1] = -2.f / sc;
     scale[2] = 2.9802322e-8f / sc;
+}
+
+// One sweep over the rows: squared norm (slightly over-estimated), the row's own power-of-two
+// scale s_i (largest magnitude to [2^13, 2^14)), rinv[i] = 1 / s_i, Yh[i, :] = fp16(Y[i, :] * s_i)
+// rounded to nearest, and the largest magnitude of the matrix (float bits, one atomicMax per CTA).
+// A row is handled by G lanes and read twice; the second read comes out of L1/L2.
+__global__ void __launch_bounds__(256) half_shadow_kernel(const float *__restrict__ Y, int64_t N, int D, int G,
+                                                          float *__restrict__ ynorm2, float *__restrict__ rinv,
+                                                          unsigned int *__restrict__ amax_bits, __half *__restrict__ Yh)
+{
+    __shared__ float wmax[8];
+    const int D4 = D >> 2;
+    const int rows_per_cta = 256 / G;
+    const int sub = threadIdx.x / G, c0 = threadIdx.x % G;
+    float cta_max = 0.f;
+    for (int64_t row = (int64_t)blockIdx.x * rows_per_cta + sub; row < N; row += (int64_t)gridDim.x * rows_per_cta) {
+        const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)row * D);
+        float s = 0.f, m = 0.f;
+        for (int c = c0; c < D4; c += 8 * G) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int cc = c + u * G;
+                v[u] = (cc < D4) ? __ldg(y4 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                s = fmaf(v[u].x, v[u].x, s);
+                s = fmaf(v[u].y, v[u].y, s);
+                s = fmaf(v[u].z, v[u].z, s);
+                s = fmaf(v[u].w, v[u].w, s);
+                m = fmaxf(fmaxf(m, fmaxf(fabsf(v[u].x), fabsf(v[u].y))), fmaxf(fabsf(v[u].z), fabsf(v[u].w)));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            if (o < G) {
+                s += __shfl_xor_sync(0xffffffffu, s, o);
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            }
+        }
+        int e = 0;
+        if (m > 0.f && m < CUDART_INF_F) frexpf(m, &e);
+        int sh = 14 - e;
+        if (sh > 100) sh = 100;
+        if (sh < -100) sh = -100;
+        const float sc = ldexpf(1.f, sh);
+        if (c0 == 0) {
+            ynorm2[row] = s * 1.0001f;
+            rinv[row] = ldexpf(1.f, -sh);
+        }
+        if (m == m && m < CUDART_INF_F) cta_max = fmaxf(cta_max, m);
+        uint2 *h4 = reinterpret_cast<uint2 *>(Yh + (size_t)row * D);
+        for (int c = c0; c < D4; c += G) {
+            const float4 v = __ldg(y4 + c);
+            const __half2 lo = __floats2half2_rn(v.x * sc, v.y * sc);
+            const __half2 hi = __floats2half2_rn(v.z * sc, v.w * sc);
+            uint2 o2;
+            o2.x = *reinterpret_cast<const unsigned int *>(&lo);
+            o2.y = *reinterpret_cast<const unsigned int *>(&hi);
+            h4[c] = o2;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cta_max = fmaxf(cta_max, __shfl_xor_sync(0xffffffffu, cta_max, o));
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = cta_max;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < 8; ++w) t = fmaxf(t, wmax[w]);
+        atomicMax(amax_bits, __float_as_uint(t));
+    }
 }
 
 // dst = fp16(src * scale[0]), round to nearest; n4 = number of float4 groups
@@ -1024,19 +1103,18 @@ cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaS
 cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, float *scale, void *Yh,
                                cudaStream_t s)
 {
+    float *rinv = scale + 4;
     cudaError_t e = cudaMemsetAsync(scale, 0, 4 * sizeof(float), s);
     if (e != cudaSuccess) return e;
-    const int threads = 256;
     const int G = lanes_per_row(D);
-    const int64_t blocks = (N * G + threads - 1) / threads;
-    row_norms_kernel<<<(unsigned)blocks, threads, 0, s>>>(Y, N, D, G, ynorm2, reinterpret_cast<unsigned int *>(scale));
+    const int rows_per_cta = 256 / G;
+    int64_t blocks = (N + rows_per_cta - 1) / rows_per_cta;
+    const int64_t cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    half_shadow_kernel<<<(unsigned)blocks, 256, 0, s>>>(Y, N, D, G, ynorm2, rinv, reinterpret_cast<unsigned int *>(scale),
+                                                        reinterpret_cast<__half *>(Yh));
     half_scale_kernel<<<1, 32, 0, s>>>(scale);
-    const size_t n4 = (size_t)N * D / 4;
-    size_t cb = (n4 + threads - 1) / threads;
-    if (cb > (size_t)sm_count() * 16) cb = (size_t)sm_count() * 16;
-    to_half_kernel<<<(unsigned)cb, threads, 0, s>>>(reinterpret_cast<const float4 *>(Y), n4, scale,
-                                                    reinterpret_cast<uint2 *>(Yh));
-    count_launch(3);
+    count_launch(2);
     return cudaGetLastError();
 }
 

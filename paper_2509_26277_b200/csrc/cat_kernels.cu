@@ -526,7 +526,7 @@ template <bool AFFINE>
 __global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
     const float *__restrict__ Y, int64_t N, int D, int K, const float *__restrict__ C, int32_t *labels,
     const int32_t *__restrict__ cand_rows, const uint64_t *__restrict__ cand_list, Control *ctl,
-    const float *gamma, const float *beta, float *out)
+    const float *gamma, const float *beta, float *out, bool fast_output_valid)
 {
     int count = ctl->cand_count;
     if ((int64_t)count > N) count = (int)N;
@@ -580,8 +580,12 @@ __global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
             }
         }
         if (bk >= K) bk = (cand[0] >= 0) ? cand[0] : 0;   // only when every distance is NaN
+        // The fast pass has already written this row's output with the label it left in
+        // labels[row]; the row is rewritten only when the exact label differs.
+        const int fast = labels[row];
+        __syncwarp();
         if (lane == 0) labels[row] = bk;
-        if (AFFINE) {
+        if (AFFINE && (bk != fast || !fast_output_valid)) {
             const float *g = gamma + (size_t)bk * D;
             const float *bb = beta + (size_t)bk * D;
             float *o = out + (size_t)row * D;
@@ -599,10 +603,10 @@ cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, co
     int blocks = (int)(want < 1184 ? want : 1184);
     if (out)
         refine_candidates_kernel<true><<<blocks, RC_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows,
-                                                                    cand_list, ctl, gamma, beta, out);
+                                                                    cand_list, ctl, gamma, beta, out, true);
     else
         refine_candidates_kernel<false><<<blocks, RC_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows,
-                                                                     cand_list, ctl, gamma, beta, out);
+                                                                     cand_list, ctl, gamma, beta, out, false);
     count_launch();
     return cudaGetLastError();
 }

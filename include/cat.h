@@ -23,8 +23,8 @@
  *     never throws, aborts or traps.
  *   - Inputs must be finite.  Non-finite values give unspecified labels but
  *     never an out-of-range label or an invalid memory access.
- *   - Limits: 1 <= K <= CAT_MAX_K, K <= N < 2^31, 1 <= D <= CAT_MAX_D.
- *     D % 4 != 0 is supported through scalar loads (slower).
+ *   - Limits: 1 <= K <= CAT_MAX_K, K <= N < 2^31 (cat_fit and the step-level sums:
+ *     N < 2^30), 1 <= D <= CAT_MAX_D.  D % 4 != 0 is supported through scalar loads (slower).
  */
 #ifndef CAT_H_
 #define CAT_H_

@@ -191,7 +191,7 @@ size_t cat_apply_workspace_bytes(int64_t N, int32_t D, int32_t K)
 
 size_t cat_fit_workspace_bytes(int64_t N, int32_t D, int32_t K)
 {
-    if (check_shape(N, D, K, false) != CAT_OK) return 0;
+    if (check_shape(N, D, K, false) != CAT_OK || N >= ((int64_t)1 << 30)) return 0;
     return carve_fit(nullptr, N, D, K).bytes;
 }
 
@@ -253,6 +253,7 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     cat_status_t st = check_shape(N, D, K, true);
     if (st != CAT_OK) return st;
     if (iters < 0) return CAT_ERR_SHAPE;
+    if (N >= ((int64_t)1 << 30)) return CAT_ERR_UNSUPPORTED;   // a round may sort 2N entries with 32-bit positions
     if (!aligned16(Yq) || !aligned16(Yfp) || !aligned16(centroids_out) || !aligned16(gamma_out) ||
         !aligned16(beta_out) || (labels_out && !aligned16(labels_out)) ||
         (init_centroids && !aligned16(init_centroids)) || (diag && !aligned16(diag)))
@@ -344,6 +345,7 @@ cat_status_t cat_cluster_sums(const float *Y, const int32_t *labels, int64_t N, 
     if (st != CAT_OK) return st;
     if (!aligned16(Y) || !aligned16(labels) || !aligned16(sums_out) || !aligned16(counts_out))
         return CAT_ERR_ALIGN;
+    if (N >= ((int64_t)1 << 30)) return CAT_ERR_UNSUPPORTED;
     if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
         return CAT_ERR_WORKSPACE;
     FitWs w = carve_fit(workspace, N, D, K);
@@ -375,6 +377,7 @@ cat_status_t cat_centred_moments(const float *Yq, const float *Yfp, const int32_
     if (!aligned16(Yq) || !aligned16(Yfp) || !aligned16(labels) || !aligned16(meanQ) ||
         !aligned16(meanF) || !aligned16(var_out) || !aligned16(cov_out))
         return CAT_ERR_ALIGN;
+    if (N >= ((int64_t)1 << 30)) return CAT_ERR_UNSUPPORTED;
     if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
         return CAT_ERR_WORKSPACE;
     FitWs w = carve_fit(workspace, N, D, K);

@@ -46,6 +46,9 @@ def test_workspace_queries_are_pure_host_functions():
     assert 262_144 * 1024 * 2 < big < 262_144 * 1024 * 2 + 128 * 2 ** 20
     assert L.cat_apply_host_workspace_bytes(4_194_304, 1024, 256) < 2 ** 30
     assert L.cat_fit_host_workspace_bytes(1024, 1000, 8) > 2 * 1024 * 1000 * 4
+    # cat_fit sorts up to 2N entries with 32-bit positions: N < 2^30
+    assert L.cat_fit_workspace_bytes(2 ** 30, 4, 2) == 0 and L.cat_fit_workspace_bytes(2 ** 30 - 1, 4, 2) > 0
+    assert L.cat_apply_workspace_bytes(2 ** 31 - 1, 4, 2) > 0
     # unsupported or nonsensical sizes give 0
     assert L.cat_apply_workspace_bytes(10, 4, binding.MAX_K + 1) == 0
     assert L.cat_apply_workspace_bytes(10, binding.MAX_D + 1, 2) == 0

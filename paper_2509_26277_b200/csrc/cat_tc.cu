@@ -718,17 +718,19 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             // ------------------------------------------------------------ MMA issuer
             if (lane == 0 && rank == 0) {
                 const uint32_t idesc = make_idesc(PAIR ? 2 * TC_BM : TC_BM, p.npad, HALF ? 0u : 2u);
-                uint32_t it = 0, ti = 0;
+                int sa = 0, sb = 0;
+                uint32_t pha = 0, phb = 0, ti = 0, it = 0;
                 bool ok = true;
                 for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
                     const int b = ti & 1;
                     if (!mbar_wait(smem_u32(&sh.tmem_empty[b]), ((ti >> 1) & 1u) ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t acc = tmem_base + (uint32_t)(b * p.npad);
-                    for (int sl = 0; sl < nslabs; ++sl, ++it) {
-                        const int sa = it % na, sb = it % nb;
-                        if (!mbar_wait(smem_u32(&sh.b_full[sb]), (it / nb) & 1u, abort_flag, p.ctl)) { ok = false; break; }
-                        if (!mbar_wait(smem_u32(&sh.a_full[sa]), (it / na) & 1u, abort_flag, p.ctl)) { ok = false; break; }
+                    for (int sl = 0; sl < nslabs; ++sl) {
+                        // ring positions and phases are carried along (no division in this loop: the
+                        // issuing thread's own instruction count is what paces the MMAs)
+                        if (!mbar_wait(smem_u32(&sh.b_full[sb]), phb, abort_flag, p.ctl)) { ok = false; break; }
+                        if (!mbar_wait(smem_u32(&sh.a_full[sa]), pha, abort_flag, p.ctl)) { ok = false; break; }
                         if (sl == 0) TC_TRACE(ti, 2);
                         if (sl == nslabs - 1) TC_TRACE(ti, 3);
                         tc_fence_after();
@@ -752,6 +754,18 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         } else {
                             tc_commit(smem_u32(&sh.a_empty[sa]));
                             tc_commit(smem_u32(&sh.b_empty[sb]));
+                        }
+                        if (AFFINE) {
+                            // (the 24-register budget of this warp in the affine kernel has no room for
+                            // the carried positions; the MMAs are not what bounds that kernel)
+                            ++it;
+                            sa = (int)(it % (uint32_t)na);
+                            pha = (it / (uint32_t)na) & 1u;
+                            sb = (int)(it % (uint32_t)nb);
+                            phb = (it / (uint32_t)nb) & 1u;
+                        } else {
+                            if (++sa == na) { sa = 0; pha ^= 1u; }
+                            if (++sb == nb) { sb = 0; phb ^= 1u; }
                         }
                     }
                     if (ok) {

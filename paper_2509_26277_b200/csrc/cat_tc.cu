@@ -652,7 +652,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         if (warp == 0) {
             // ------------------------------------------------------------ TMA producer
             if (lane == 0) {
-                uint32_t it = 0, ti = 0;
+                uint32_t ti = 0, ph = 0;
+                int s = 0;   // ring position and phase, carried along
                 bool ok = true;
                 for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
                     const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
@@ -660,9 +661,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         // at most one tile ahead of the streaming warps: tile ti - 2 is streamed out
                         if (!wait_progress(&sh.rows_streamed, (int)(ti - 1) * TC_BM, abort_flag, p.ctl)) { ok = false; break; }
                     }
-                    for (int sl = 0; sl < nslabs; ++sl, ++it) {
-                        const int s = it % na;
-                        const uint32_t ph = (it / na) & 1u;
+                    for (int sl = 0; sl < nslabs; ++sl) {
                         if (!mbar_wait(smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
                         if (sl == 0) TC_TRACE(ti, 0);
                         if (sl == nslabs - 1) TC_TRACE(ti, 1);
@@ -677,6 +676,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                             mbar_arrive_expect_tx(full, (uint32_t)TC_A_BYTES);
                             tma_load_2d(a_dst, &mapA, full, sl * BK, (int)row0);
                         }
+                        if (++s == na) { s = 0; ph ^= 1u; }
                     }
                 }
                 if (!ok && rank == 0) {
@@ -689,12 +689,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         } else if (warp == 2) {
             // ------------------------------------------------------------ TMA producer, centroid slabs
             if (lane == 0) {
-                uint32_t it = 0;
+                uint32_t ph = 0;
+                int s = 0;
                 bool ok = true;
                 for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step) {
-                    for (int sl = 0; sl < nslabs; ++sl, ++it) {
-                        const int s = it % nb;
-                        const uint32_t ph = (it / nb) & 1u;
+                    for (int sl = 0; sl < nslabs; ++sl) {
                         if (!mbar_wait(smem_u32(&sh.b_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
                         const uint32_t b_dst = b_base + (uint32_t)(s * b_bytes);
                         if (PAIR) {
@@ -706,6 +705,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                             mbar_arrive_expect_tx(full, (uint32_t)b_bytes);
                             tma_load_2d(b_dst, &mapB, full, sl * BK, 0);
                         }
+                        if (++s == nb) { s = 0; ph ^= 1u; }
                     }
                 }
                 if (!ok && rank == 0) {
@@ -718,6 +718,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             // ------------------------------------------------------------ MMA issuer
             if (lane == 0 && rank == 0) {
                 const uint32_t idesc = make_idesc(PAIR ? 2 * TC_BM : TC_BM, p.npad, HALF ? 0u : 2u);
+                const uint64_t adesc0 = AFFINE ? 0 : make_smem_desc(tiles_base), bdesc0 = AFFINE ? 0 : make_smem_desc(b_base);
                 int sa = 0, sb = 0;
                 uint32_t pha = 0, phb = 0, ti = 0, it = 0;
                 bool ok = true;
@@ -734,8 +735,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         if (sl == 0) TC_TRACE(ti, 2);
                         if (sl == nslabs - 1) TC_TRACE(ti, 3);
                         tc_fence_after();
-                        const uint64_t adesc = make_smem_desc(tiles_base + (uint32_t)(sa * TC_A_BYTES));
-                        const uint64_t bdesc = make_smem_desc(b_base + (uint32_t)(sb * b_bytes));
+                        // (the start address sits in the low bits of the descriptor, in 16-byte units)
+                        const uint64_t adesc = AFFINE ? make_smem_desc(tiles_base + (uint32_t)(sa * TC_A_BYTES))
+                                                      : adesc0 + (uint64_t)(uint32_t)(sa * (TC_A_BYTES >> 4));
+                        const uint64_t bdesc = AFFINE ? make_smem_desc(b_base + (uint32_t)(sb * b_bytes))
+                                                      : bdesc0 + (uint64_t)(uint32_t)(sb * (b_bytes >> 4));
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk) {   // 8 tf32 or 16 f16 = 32 B per MMA: +2 in 16-byte units
                             const uint32_t accum = (sl > 0 || kk > 0) ? 1u : 0u;

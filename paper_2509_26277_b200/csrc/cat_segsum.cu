@@ -382,14 +382,14 @@ __global__ void segment_combine3_kernel(const double *__restrict__ part, const i
 // K + k); c_k = float(S_k / n_k) where n_k > 0; and for the next assignment the squared norm
 // of c_k (fp64, rounded up), optionally the fp16 copy fp16(c_k * scale[0]), and the reset of the
 // exact-pass queues.
-__global__ void __launch_bounds__(256) centroid_update_kernel(const double *__restrict__ part,
+__global__ void __launch_bounds__(1024) centroid_update_kernel(const double *__restrict__ part,
                                                               const int32_t *__restrict__ seg_start,
                                                               const int64_t *__restrict__ counts, int D, int K,
                                                               double *__restrict__ sums, float *__restrict__ C,
                                                               float *__restrict__ cnorm, const float *__restrict__ scale,
                                                               __half *__restrict__ Ch, Control *ctl)
 {
-    __shared__ double red[8];
+    __shared__ double red[32];
     const int k = blockIdx.x;
     if (k == 0 && threadIdx.x == 0) {
         ctl->refine_count = 0;
@@ -420,7 +420,7 @@ __global__ void __launch_bounds__(256) centroid_update_kernel(const double *__re
     __syncthreads();
     if (threadIdx.x == 0) {
         double t = 0.0;
-        for (int w = 0; w < 8; ++w) t += red[w];
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
         cnorm[k] = __double2float_ru(t);
     }
 }
@@ -538,7 +538,9 @@ cudaError_t launch_centroid_update(const double *part, const int32_t *seg_start,
                                    int K, double *sums, float *C, float *cnorm, const float *scale, void *Ch,
                                    Control *ctl, cudaStream_t s)
 {
-    centroid_update_kernel<<<K, 256, 0, s>>>(part, seg_start, counts, D, K, sums, C, cnorm, scale,
+    // one thread per column where the row is short enough: the loads of a column depend on each other
+    const int threads = D >= 1024 ? 1024 : (D >= 512 ? 512 : 256);
+    centroid_update_kernel<<<K, threads, 0, s>>>(part, seg_start, counts, D, K, sums, C, cnorm, scale,
                                              reinterpret_cast<__half *>(Ch), ctl);
     count_launch();
     return cudaGetLastError();

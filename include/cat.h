@@ -232,6 +232,14 @@ cat_status_t cat_fit_host(const float *Yq_host, const float *Yfp_host, int64_t N
 cat_status_t cat_workspace_report(const void *workspace, void *stream, int64_t *refined_last_host,
                                   int64_t *refined_total_host, int32_t *device_status_host);
 
+/* Self-test of the failure path of the device-side waits.  The tensor-core kernels wait on
+ * barriers with a time limit; a wait that runs out records CAT_ERR_DEVICE_TIMEOUT in the
+ * workspace's control block and the kernel returns instead of hanging.  This call enqueues one
+ * warp that waits limit_ms (clamped to 1 .. 1000) on a barrier nothing completes; afterwards
+ * cat_workspace_report on the same workspace gives device_status = CAT_ERR_DEVICE_TIMEOUT.
+ * Any workspace of at least 256 bytes will do; its counters are reset. */
+cat_status_t cat_selftest_wait_timeout(void *workspace, size_t workspace_bytes, int32_t limit_ms, void *stream);
+
 /* Kernel selection for the distance contraction.  With K >= min_k (and D % 4 == 0,
  * K <= 256) the scores are formed on the tensor cores (tcgen05, TF32 operands, fp32
  * accumulation); below it on the fp32 pipes.  Either way undecided rows are settled in

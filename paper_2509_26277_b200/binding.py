@@ -30,6 +30,7 @@ EXPORTS = [
     "cat_centroids_from_sums",
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
+    "cat_selftest_wait_timeout",
     "cat_set_tensor_core_min_k", "cat_get_tensor_core_min_k", "cat_status_string",
     "cat_last_cuda_error", "cat_version", "cat_kernel_launches",
 ]
@@ -91,6 +92,8 @@ def lib():
                  "cat_cluster_sums", "cat_centroids_from_sums", "cat_centred_moments",
                  "cat_solve_gamma_beta", "cat_apply_host", "cat_fit_host"):
         getattr(L, name).restype = ctypes.c_int
+    L.cat_selftest_wait_timeout.argtypes = [vp, sz, i32, vp]
+    L.cat_selftest_wait_timeout.restype = ctypes.c_int
     L.cat_workspace_report.argtypes = [vp, vp, vp, vp, vp]
     L.cat_workspace_report.restype = ctypes.c_int
     L.cat_set_tensor_core_min_k.argtypes = [i32]
@@ -344,6 +347,13 @@ def cat_fit_host(Yq_host, Yfp_host, K: int, iters: int, C_host, G_host, B_host, 
                             ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream())
     _check(st, "cat_fit_host")
     return C_host, G_host, B_host
+
+
+def cat_selftest_wait_timeout(ws, limit_ms: int = 20) -> None:
+    """Enqueue the bounded-wait self-test on workspace `ws` (see cat.h); read the outcome with
+    cat_workspace_report."""
+    _check(lib().cat_selftest_wait_timeout(ctypes.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size(),
+                                           int(limit_ms), _stream()), "cat_selftest_wait_timeout")
 
 
 def cat_workspace_report(ws) -> dict:

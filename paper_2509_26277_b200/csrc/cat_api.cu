@@ -414,6 +414,16 @@ cat_status_t cat_workspace_report(const void *workspace, void *stream, int64_t *
     return CAT_OK;
 }
 
+cat_status_t cat_selftest_wait_timeout(void *workspace, size_t workspace_bytes, int32_t limit_ms, void *stream)
+{
+    if (!workspace) return CAT_ERR_NULL;
+    if (!aligned16(workspace) || workspace_bytes < sizeof(Control)) return CAT_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    CAT_CUDA(launch_reset_control(reinterpret_cast<Control *>(workspace), s));
+    CAT_CUDA(launch_wait_selftest(reinterpret_cast<Control *>(workspace), limit_ms, s));
+    return CAT_OK;
+}
+
 void cat_set_tensor_core_min_k(int32_t min_k)
 {
     g_tc_min_k.store(min_k < 1 ? 1 : min_k, std::memory_order_relaxed);

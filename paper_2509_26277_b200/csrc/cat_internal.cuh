@@ -108,6 +108,9 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
                              const float *gamma, const float *beta, float *out, cudaStream_t s,
                              const void *Yh = nullptr, const void *Ch = nullptr, const float *scale = nullptr);
 
+// One warp waits (at most limit_ms, clamped to 1 .. 1000) on a barrier that is never completed.
+cudaError_t launch_wait_selftest(Control *ctl, int limit_ms, cudaStream_t s);
+
 // fp16 copy of a matrix for repeated assignments, made in one sweep: squared row norms, per-row
 // power-of-two scales, Yh[i] = fp16(Y[i] * scale_i), and scale[4 + N] = {centroid scale s_c from the
 // largest magnitude, -2 / s_c, 2^-25 / s_c, unused, then 1 / scale_i for every row}.  Needs D % 8 == 0.

@@ -115,7 +115,8 @@ __device__ __forceinline__ uint64_t global_timer()
 // Bounded wait.  Returns false after a timeout or once another role has given up.
 // (Inlined on purpose: a called function inside the re-divided register budgets of the
 // affine kernel sends ptxas into a very long compile.)
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, Control *ctl)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, Control *ctl,
+                                          uint64_t limit_ns = TC_TIMEOUT_NS)
 {
     uint64_t t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -125,7 +126,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             uint64_t now = global_timer();
             if (t0 == 0) {
                 t0 = now;
-            } else if (now - t0 > TC_TIMEOUT_NS) {
+            } else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicExch(&ctl->device_status, (int)CAT_ERR_DEVICE_TIMEOUT);
                 return false;
@@ -1033,6 +1034,24 @@ __global__ void to_half_kernel(const float4 *__restrict__ src, size_t n4, const 
     }
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes, with
+// the given limit; the wait gives up, records CAT_ERR_DEVICE_TIMEOUT and the kernel returns.
+__global__ void wait_selftest_kernel(Control *ctl, uint64_t limit_ns)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    {
+        const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, ctl, limit_ns);
+        (void)ok;
+    }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -1145,6 +1164,15 @@ cudaError_t launch_to_half(const float *src, size_t n, const float *scale, void 
     if (cb < 1) cb = 1;
     to_half_kernel<<<(unsigned)cb, threads, 0, s>>>(reinterpret_cast<const float4 *>(src), n4, scale,
                                                     reinterpret_cast<uint2 *>(dst));
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_wait_selftest(Control *ctl, int limit_ms, cudaStream_t s)
+{
+    if (limit_ms < 1) limit_ms = 1;
+    if (limit_ms > 1000) limit_ms = 1000;
+    wait_selftest_kernel<<<1, 32, 0, s>>>(ctl, (uint64_t)limit_ms * 1000000ull);
     count_launch();
     return cudaGetLastError();
 }

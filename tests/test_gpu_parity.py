@@ -344,3 +344,18 @@ def test_non_default_stream_and_missing_labels_out():
         out = B.cat_apply(Yq, C, torch.ones_like(C), torch.zeros_like(C))
     s.synchronize()
     assert torch.equal(a, B.cat_assign(Yq, C)) and torch.equal(out, Yq)
+
+
+def test_bounded_device_wait_reports_a_timeout_and_leaves_the_context_usable():
+    """A device-side wait that can never be satisfied gives up after its limit: the kernel returns,
+    the status word says CAT_ERR_DEVICE_TIMEOUT, and the next call on the same workspace works."""
+    Yq = dev(_rand(21, 1000, 256))
+    C = dev(_rand(22, 40, 256))
+    ws = B.workspace("apply", 1000, 256, 40, "cuda")
+    B.cat_selftest_wait_timeout(ws, limit_ms=20)
+    rep = B.cat_workspace_report(ws)
+    assert rep["device_status"] == 6
+    labels = B.cat_assign(Yq, C, ws=ws)
+    assert B.cat_workspace_report(ws)["device_status"] == 0
+    lab, best, second = O.assign(host(Yq), host(C))
+    labels_match(host(labels), lab, best, second, "labels after the self-test")

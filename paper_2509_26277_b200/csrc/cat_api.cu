@@ -59,7 +59,7 @@ FitWs carve_fit(void *base, int64_t N, int D, int K)
     w.blk_hist = c.take<uint32_t>((size_t)g.nblk * 2 * K);
     w.key_total = c.take<uint32_t>((size_t)2 * K);
     w.cluster_start = c.take<int32_t>((size_t)2 * K + 1);
-    w.seg_start = c.take<int32_t>((size_t)2 * K + 1);
+    w.seg_start = c.take<int32_t>((size_t)2 * K + 2);
     w.order = c.take<int32_t>((size_t)2 * N);
     w.labels_prev = c.take<int32_t>((size_t)N);
     {

@@ -41,7 +41,7 @@ struct Control {
 // at launch time.
 struct SegGeom {
     int nblk;       // 1024-entry blocks of the sort
-    int seg_rows;   // rows per segment (multiple of 128)
+    int seg_rows;   // largest rows per segment (multiple of 128); a sort may choose shorter segments
     int max_segs;   // upper bound on the number of segments: ceil(NE / seg_rows) + KK
 };
 SegGeom seg_geometry(int64_t NE, int D, int KK);
@@ -66,7 +66,7 @@ struct FitWs {
     uint32_t *blk_hist;    // [nblk][2K] key histogram / offsets of the sort
     uint32_t *key_total;   // [2K] entries per key
     int32_t *cluster_start; // [2K+1] first position of each key in `order`
-    int32_t *seg_start;    // [2K+1] first segment of each key
+    int32_t *seg_start;    // [2K+2] first segment of each key, total, segment length of the current sort
     int32_t *order;        // [2N] row indices sorted by key (stable)
     int32_t *labels_prev;  // [N] labels of the previous Lloyd round
     double *segpart;       // [max_segs][2][D] per-segment partial sums

@@ -90,48 +90,70 @@ __global__ void __launch_bounds__(256) label_scan_blocks_kernel(uint32_t *__rest
     if (lane == 0) key_total[k] = carry;
 }
 
-// One CTA of 1024 threads (KK <= 1024): exclusive scans of the key totals (cluster_start) and
-// of the segment counts ceil(total / seg_rows) (seg_start), KK + 1 entries each; cluster sizes:
-// full mode counts[k] = total[k]; delta mode counts[k] += total[k] - total[K + k].
+// Exclusive scan over the 1024 threads of the CTA (one value per thread); returns the exclusive
+// prefix of the calling thread and, through `total`, the sum of all values.
+__device__ __forceinline__ uint32_t cta_exclusive_scan(uint32_t v, uint32_t *wsum /*[33] shared*/, uint32_t &total)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint32_t incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();   // wsum may still be read from an earlier scan
+    if (lane == 31) wsum[w] = incl;
+    __syncthreads();
+    if (w == 0) {
+        const uint32_t a = wsum[lane];
+        uint32_t x = a;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += t;
+        }
+        wsum[lane] = x - a;   // exclusive
+        if (lane == 31) wsum[32] = x;
+    }
+    __syncthreads();
+    total = wsum[32];
+    return wsum[w] + incl - v;
+}
+
+// One CTA of 1024 threads (KK <= 1024): exclusive scan of the key totals (cluster_start, KK + 1
+// entries), the segment length for this sort, the exclusive scan of the segment counts
+// ceil(total / length) (seg_start, KK + 1 entries, followed by the length itself), and the cluster
+// sizes: full mode counts[k] = total[k]; delta mode counts[k] += total[k] - total[K + k].
+// The segment length shrinks with the number of entries M actually present (a delta sort of a
+// settled clustering holds a handful): length = seg_rows_max * M / NE rounded up to 16, at least 16,
+// so that short lists still spread over many CTAs and the segment count stays within
+// NE / seg_rows_max + KK.
 __global__ void __launch_bounds__(1024) label_scan_keys_kernel(const uint32_t *__restrict__ key_total, int K, int KK,
-                                                                int seg_rows, int delta, int64_t *__restrict__ counts,
+                                                                int seg_rows_max, int64_t NE, int delta,
+                                                                int64_t *__restrict__ counts,
                                                                 int32_t *__restrict__ cluster_start,
                                                                 int32_t *__restrict__ seg_start)
 {
-    __shared__ uint32_t wsum_a[32], wsum_s[32];
-    const int k = threadIdx.x, lane = k & 31, w = k >> 5;
+    __shared__ uint32_t wsum[33];
+    const int k = threadIdx.x;
     const uint32_t tot = (k < KK) ? key_total[k] : 0u;
-    const uint32_t sg = (tot + (uint32_t)seg_rows - 1) / (uint32_t)seg_rows;
-    uint32_t ia = tot, is = sg;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o);
-        const uint32_t ts = __shfl_up_sync(0xffffffffu, is, o);
-        if (lane >= o) { ia += ta; is += ts; }
-    }
-    if (lane == 31) { wsum_a[w] = ia; wsum_s[w] = is; }
-    __syncthreads();
-    if (w == 0) {
-        uint32_t a = wsum_a[lane], sgs = wsum_s[lane];
-        uint32_t xa = a, xs = sgs;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t ta = __shfl_up_sync(0xffffffffu, xa, o);
-            const uint32_t ts = __shfl_up_sync(0xffffffffu, xs, o);
-            if (lane >= o) { xa += ta; xs += ts; }
-        }
-        wsum_a[lane] = xa - a;   // exclusive
-        wsum_s[lane] = xs - sgs;
-    }
-    __syncthreads();
-    const uint32_t ea = wsum_a[w] + ia - tot, es = wsum_s[w] + is - sg;
+    uint32_t M = 0;
+    const uint32_t ea = cta_exclusive_scan(tot, wsum, M);
+    int64_t sr = ((int64_t)seg_rows_max * (int64_t)M + NE - 1) / NE;
+    sr = (sr + 15) / 16 * 16;
+    if (sr < 16) sr = 16;
+    if (sr > seg_rows_max) sr = seg_rows_max;
+    const uint32_t sg = (tot + (uint32_t)sr - 1) / (uint32_t)sr;
+    uint32_t nseg = 0;
+    const uint32_t es = cta_exclusive_scan(sg, wsum, nseg);
     if (k < KK) {
         cluster_start[k] = (int32_t)ea;
         seg_start[k] = (int32_t)es;
-        if (k == KK - 1) {
-            cluster_start[KK] = (int32_t)(ea + tot);
-            seg_start[KK] = (int32_t)(es + sg);
-        }
+    }
+    if (k == 0) {
+        cluster_start[KK] = (int32_t)M;
+        seg_start[KK] = (int32_t)nseg;
+        seg_start[KK + 1] = (int32_t)sr;
     }
     if (k < K) {
         if (delta) counts[k] += (int64_t)tot - (int64_t)key_total[K + k];
@@ -241,9 +263,10 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
         if (p.seg_start[mid] <= seg) lo = mid; else hi = mid;
     }
     const int k = lo;
-    const int first = p.cluster_start[k] + (seg - p.seg_start[k]) * p.seg_rows;
+    const int seg_rows = p.seg_start[p.K + 1];   // length chosen by the sort for this list
+    const int first = p.cluster_start[k] + (seg - p.seg_start[k]) * seg_rows;
     int nrows = p.cluster_start[k + 1] - first;
-    if (nrows > p.seg_rows) nrows = p.seg_rows;
+    if (nrows > seg_rows) nrows = seg_rows;
 
     const int tid = threadIdx.x;
     const int tpr = p.tpr;
@@ -455,8 +478,8 @@ cudaError_t launch_label_sort(const int32_t *labels, const int32_t *prev, int64_
     const int KK = prev ? 2 * K : K;
     label_hist_kernel<<<g.nblk, SORT_BLOCK, (size_t)KK * sizeof(uint32_t), s>>>(labels, prev, N, K, KK, blk_hist);
     label_scan_blocks_kernel<<<(KK * 32 + 255) / 256, 256, 0, s>>>(blk_hist, g.nblk, KK, key_total);
-    label_scan_keys_kernel<<<1, 1024, 0, s>>>(key_total, K, KK, g.seg_rows, prev ? 1 : 0, counts, cluster_start,
-                                               seg_start);
+    label_scan_keys_kernel<<<1, 1024, 0, s>>>(key_total, K, KK, g.seg_rows, prev ? 2 * N : N, prev ? 1 : 0, counts,
+                                               cluster_start, seg_start);
     const size_t sc_smem = (size_t)32 * KK * sizeof(uint16_t);
     if (sc_smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(label_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

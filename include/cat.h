@@ -248,6 +248,17 @@ cat_status_t cat_selftest_wait_timeout(void *workspace, size_t workspace_bytes, 
 void cat_set_tensor_core_min_k(int32_t min_k);
 int32_t cat_get_tensor_core_min_k(void);
 
+/* Kernel selection for the fused inference kernel (tensor-core path, D >= 128).  Two forms
+ * compute the same thing: row tiles (a CTA pair shares 256 rows, each CTA all D columns of its
+ * 128), and column split (the cs CTAs of a cluster share 128 rows, each staging D / cs columns;
+ * the partial scores are summed through distributed shared memory).  The second keeps fewer
+ * bytes in flight between a row's two reads, which pays once N x D no longer fits in L2.
+ * cs = 0: chosen from the shape (default); 1: never split; 2 or 4: split over that many CTAs
+ * wherever the shape allows it (D a multiple of 32 cs, K rounded up to 32 cs at most 256,
+ * N > 128), row tiles elsewhere.  Other values count as 0.  Process-wide setting. */
+void cat_set_apply_column_split(int32_t cs);
+int32_t cat_get_apply_column_split(void);
+
 const char *cat_status_string(cat_status_t status);
 int cat_last_cuda_error(void);           /* cudaError_t of the last failing runtime call on this thread */
 const char *cat_version(void);

@@ -31,7 +31,8 @@ EXPORTS = [
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
     "cat_selftest_wait_timeout",
-    "cat_set_tensor_core_min_k", "cat_get_tensor_core_min_k", "cat_status_string",
+    "cat_set_tensor_core_min_k", "cat_get_tensor_core_min_k",
+    "cat_set_apply_column_split", "cat_get_apply_column_split", "cat_status_string",
     "cat_last_cuda_error", "cat_version", "cat_kernel_launches",
 ]
 
@@ -99,6 +100,9 @@ def lib():
     L.cat_set_tensor_core_min_k.argtypes = [i32]
     L.cat_set_tensor_core_min_k.restype = None
     L.cat_get_tensor_core_min_k.restype = i32
+    L.cat_set_apply_column_split.argtypes = [i32]
+    L.cat_set_apply_column_split.restype = None
+    L.cat_get_apply_column_split.restype = i32
     L.cat_status_string.argtypes = [ctypes.c_int]
     L.cat_status_string.restype = ctypes.c_char_p
     L.cat_last_cuda_error.restype = ctypes.c_int
@@ -371,6 +375,14 @@ def cat_set_tensor_core_min_k(min_k: int) -> None:
 
 def cat_get_tensor_core_min_k() -> int:
     return int(lib().cat_get_tensor_core_min_k())
+
+
+def cat_set_apply_column_split(cs: int) -> None:
+    lib().cat_set_apply_column_split(int(cs))
+
+
+def cat_get_apply_column_split() -> int:
+    return int(lib().cat_get_apply_column_split())
 
 
 def cat_version() -> str:

@@ -431,6 +431,10 @@ void cat_set_tensor_core_min_k(int32_t min_k)
 
 int32_t cat_get_tensor_core_min_k(void) { return g_tc_min_k.load(std::memory_order_relaxed); }
 
+void cat_set_apply_column_split(int32_t cs) { set_apply_column_split((int)cs); }
+
+int32_t cat_get_apply_column_split(void) { return (int32_t)get_apply_column_split(); }
+
 const char *cat_status_string(cat_status_t status)
 {
     switch (status) {

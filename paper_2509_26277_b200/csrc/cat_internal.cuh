@@ -100,6 +100,9 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
 
 // Tensor-core (tcgen05, TF32) variant of launch_assign; ynorm2 is needed when out == nullptr.
 bool tc_supported(int64_t N, int D, int K);
+// Column-split form of the fused inference kernel: 0 = chosen by shape, 1 = never, 2 / 4 = that cluster size where it applies.
+void set_apply_column_split(int cs);
+int get_apply_column_split();
 cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaStream_t s);
 // With Yh / Ch / scale (labels only): the fp16 copies of the rows and centroids are the MMA operands.
 cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,

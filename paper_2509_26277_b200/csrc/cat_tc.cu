@@ -37,6 +37,8 @@
 // returns.
 #include "cat_internal.cuh"
 
+#include <atomic>
+
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
@@ -884,6 +886,387 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     }
 }
 
+// ------------------------------------------------------------------ column-split inference kernel
+//
+// The bytes between a row's first read (TMA, for the MMA) and its second (the streaming warps)
+// decide whether the second read still finds the row in L2, and they grow with the rows a CTA
+// has in flight.  Here the CS CTAs of a cluster share ONE 128-row tile: CTA c stages columns
+// [c D / CS, (c + 1) D / CS) of the rows and of ALL centroids and accumulates partial dot
+// products (cta_group::1, M = 128, N = K) in its own TMEM.  The partial scores are then summed
+// across the cluster through distributed shared memory: CTA c collects, for all 128 rows, the
+// partials of centroids [c W, (c + 1) W), W = npad / CS, finds the four smallest keys among
+// those, and sends them to the CTA that owns the row (rows [q 128 / CS, (q + 1) 128 / CS) belong
+// to CTA q), which merges the CS lists and streams the row out.  Per CTA only 128 / CS rows'
+// worth of bytes is in flight; the price is CS times the centroid bytes out of L2 per row.
+struct TcSplitShared {
+    uint64_t a_full[TC_MAX_A_STAGES];
+    uint64_t a_empty[TC_MAX_A_STAGES];
+    uint64_t b_full[TC_MAX_B_STAGES];
+    uint64_t b_empty[TC_MAX_B_STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t lab_full[2];
+    uint64_t lab_empty[2];
+    uint64_t x_full;              // the peers' partial scores of a tile have landed here
+    uint64_t x_empty;             // the peers have read what this CTA sent them
+    uint64_t k_full[2];           // the peers' keys of the rows this CTA owns have landed
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int rows_streamed;
+    float red[32];
+    float cn[256];
+    float4 top_key[2][TC_BM];     // merged keys of the rows this CTA owns (the first 128 / CS entries)
+    float4 peer_key[2][TC_BM];    // [buffer][source CTA * (128 / CS) + row]
+};
+
+__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// arrival on a barrier of another CTA that publishes this thread's earlier (fenced) writes to it
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_acq_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded, warp-uniform wait on a barrier that CTAs of the cluster arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, Control *ctl)
+{
+    bool ok = true;
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait_acq_cluster(bar, parity)) break;
+        if (*abort_flag) { ok = false; break; }
+        if ((it & 63u) == 63u) {
+            uint64_t now = global_timer();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > TC_TIMEOUT_NS) {
+                *abort_flag = 1;
+                atomicExch(&ctl->device_status, (int)CAT_ERR_DEVICE_TIMEOUT);
+                ok = false;
+                break;
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
+template <int CS>
+__global__ void __launch_bounds__(TC_THREADS_AFFINE, 1)
+apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p)
+{
+    constexpr int RP = TC_BM / CS;                 // rows of a tile this CTA owns
+    constexpr int OWNER_WARPS = TC_SCORE_WARPS / CS;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+    unsigned char *tiles = smem_raw + (tiles_base - raw);
+    const int b_bytes = p.npad * 128;
+    const int na = p.a_stages, nb = p.b_stages;
+    const int W = p.npad / CS;                     // centroids this CTA reduces
+    const uint32_t b_base = tiles_base + (uint32_t)(na * TC_A_BYTES);
+    const uint32_t x_base = b_base + (uint32_t)(nb * b_bytes);          // [CS - 1][128][W] fp32, 16-byte chunks swizzled
+    const int x_bytes = (CS - 1) * TC_BM * W * 4;
+    unsigned char *x_ptr = tiles + (size_t)na * TC_A_BYTES + (size_t)nb * b_bytes;
+    TcSplitShared &sh = *reinterpret_cast<TcSplitShared *>(x_ptr + x_bytes);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t crank = cluster_ctarank();
+    volatile int *abort_flag = &sh.abort_flag;
+    const int64_t num_units = (p.N + TC_BM - 1) / TC_BM;
+    const int64_t unit_first = (int64_t)(blockIdx.x / CS);
+    const int64_t unit_step = (int64_t)(gridDim.x / CS);
+    const int nslabs = p.D / (32 * CS);            // slabs of this CTA's columns
+    const int slab0 = (int)crank * nslabs;
+
+    if (tid == 0) {
+        for (int s = 0; s < na; ++s) {
+            mbar_init(smem_u32(&sh.a_full[s]), 1);
+            mbar_init(smem_u32(&sh.a_empty[s]), 1);
+        }
+        for (int s = 0; s < nb; ++s) {
+            mbar_init(smem_u32(&sh.b_full[s]), 1);
+            mbar_init(smem_u32(&sh.b_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh.tmem_full[b]), 1);
+            mbar_init(smem_u32(&sh.tmem_empty[b]), TC_SCORE_WARPS);
+            mbar_init(smem_u32(&sh.lab_full[b]), OWNER_WARPS);
+            mbar_init(smem_u32(&sh.lab_empty[b]), TC_STREAM_WARPS);
+            mbar_init(smem_u32(&sh.k_full[b]), (CS - 1) * OWNER_WARPS);
+        }
+        mbar_init(smem_u32(&sh.x_full), (CS - 1) * TC_SCORE_WARPS);
+        mbar_init(smem_u32(&sh.x_empty), (CS - 1) * TC_SCORE_WARPS);
+        mbar_init(smem_u32(&sh.drain), 1);
+        sh.abort_flag = 0;
+        sh.rows_streamed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    {
+        float m = 0.f;
+        for (int k = tid; k < 256; k += blockDim.x) {
+            float v = (k < p.K) ? p.cnorm[k] : TC_KEY_INIT;
+            sh.cn[k] = v;
+            if (k < p.K) m = fmaxf(m, v);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) sh.red[warp] = m;
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh.tmem_base), (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();   // the peers' barriers exist before anything arrives on them
+    tc_fence_after();
+    float cmax2 = 0.f;
+    for (int w2 = 0; w2 < (int)(blockDim.x >> 5); ++w2) cmax2 = fmaxf(cmax2, sh.red[w2]);
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp < TC_FIRST_SCORE_WARP) {
+        setmaxnreg_dec<TC_REGS_CONTROL>();
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer, row slabs
+            if (lane == 0) {
+                uint32_t ti = 0, ph = 0;
+                int s = 0;
+                bool ok = true;
+                for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
+                    const int row0 = (int)(unit * TC_BM);
+                    if (ti > 1) {
+                        // at most one tile ahead of the streaming warps
+                        if (!wait_progress(&sh.rows_streamed, (int)(ti - 1) * RP, abort_flag, p.ctl)) { ok = false; break; }
+                    }
+                    for (int sl = 0; sl < nslabs; ++sl) {
+                        if (!mbar_wait(smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        if (sl == 0) TC_TRACE(ti, 0);
+                        if (sl == nslabs - 1) TC_TRACE(ti, 1);
+                        const uint32_t full = smem_u32(&sh.a_full[s]);
+                        mbar_arrive_expect_tx(full, (uint32_t)TC_A_BYTES);
+                        tma_load_2d(tiles_base + (uint32_t)(s * TC_A_BYTES), &mapA, full, (slab0 + sl) * 32, row0);
+                        if (++s == na) { s = 0; ph ^= 1u; }
+                    }
+                }
+                if (!ok) {
+                    for (int s2 = 0; s2 < na; ++s2)
+                        for (int tries = 0; tries < 100000; ++tries)
+                            if (mbar_try_wait(smem_u32(&sh.a_full[s2]), 0) || mbar_try_wait(smem_u32(&sh.a_full[s2]), 1)) break;
+                }
+            }
+        } else if (warp == 2) {
+            // ------------------------------------------------------------ TMA producer, centroid slabs
+            if (lane == 0) {
+                uint32_t ph = 0;
+                int s = 0;
+                bool ok = true;
+                for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step) {
+                    for (int sl = 0; sl < nslabs; ++sl) {
+                        if (!mbar_wait(smem_u32(&sh.b_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                        const uint32_t full = smem_u32(&sh.b_full[s]);
+                        mbar_arrive_expect_tx(full, (uint32_t)b_bytes);
+                        tma_load_2d(b_base + (uint32_t)(s * b_bytes), &mapB, full, (slab0 + sl) * 32, 0);
+                        if (++s == nb) { s = 0; ph ^= 1u; }
+                    }
+                }
+                if (!ok) {
+                    for (int s2 = 0; s2 < nb; ++s2)
+                        for (int tries = 0; tries < 100000; ++tries)
+                            if (mbar_try_wait(smem_u32(&sh.b_full[s2]), 0) || mbar_try_wait(smem_u32(&sh.b_full[s2]), 1)) break;
+                }
+            }
+        } else if (warp == 1) {
+            // ------------------------------------------------------------ MMA issuer
+            if (lane == 0) {
+                const uint32_t idesc = make_idesc(TC_BM, p.npad, 2u);
+                int sa = 0, sb = 0;
+                uint32_t pha = 0, phb = 0, ti = 0;
+                bool ok = true;
+                for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
+                    const int b = ti & 1;
+                    if (!mbar_wait(smem_u32(&sh.tmem_empty[b]), ((ti >> 1) & 1u) ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t acc = tmem_base + (uint32_t)(b * p.npad);
+                    for (int sl = 0; sl < nslabs; ++sl) {
+                        if (!mbar_wait(smem_u32(&sh.b_full[sb]), phb, abort_flag, p.ctl)) { ok = false; break; }
+                        if (!mbar_wait(smem_u32(&sh.a_full[sa]), pha, abort_flag, p.ctl)) { ok = false; break; }
+                        if (sl == 0) TC_TRACE(ti, 2);
+                        if (sl == nslabs - 1) TC_TRACE(ti, 3);
+                        tc_fence_after();
+                        const uint64_t adesc = make_smem_desc(tiles_base + (uint32_t)(sa * TC_A_BYTES));
+                        const uint64_t bdesc = make_smem_desc(b_base + (uint32_t)(sb * b_bytes));
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_tf32(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
+                        tc_commit(smem_u32(&sh.a_empty[sa]));
+                        tc_commit(smem_u32(&sh.b_empty[sb]));
+                        if (++sa == na) { sa = 0; pha ^= 1u; }
+                        if (++sb == nb) { sb = 0; phb ^= 1u; }
+                    }
+                    if (ok) tc_commit(smem_u32(&sh.tmem_full[b]));
+                }
+                tc_commit(smem_u32(&sh.drain));
+                for (int tries = 0; tries < 4000000; ++tries)
+                    if (mbar_try_wait(smem_u32(&sh.drain), 0)) break;
+            }
+        }
+    } else if (warp < TC_FIRST_STREAM_WARP) {
+        // ------------------------------------------------------------ score warps
+        setmaxnreg_dec<TC_REGS_SCORE>();
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;            // row of the tile = TMEM lane
+        const uint32_t owner = (uint32_t)(r / RP);    // CTA that owns this row
+        const uint32_t swz = (uint32_t)(r & 7);
+        uint32_t ti = 0;
+        bool ok = true;
+        for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
+            const int b = ti & 1;
+            const uint32_t ph = (ti >> 1) & 1u;
+            if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
+            tc_fence_after();
+            if (quarter == 0 && lane == 0) TC_TRACE(ti, 4);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
+            uint32_t ra[16], rb[16];
+            // ---- send: the peers' centroid ranges of this CTA's partial scores
+            if (!mbar_wait_cluster_warp(smem_u32(&sh.x_empty), (ti & 1u) ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+#pragma unroll 1
+            for (uint32_t d = 1; d < (uint32_t)CS; ++d) {
+                const uint32_t q = (crank + d) % CS;                  // destination CTA
+                const uint32_t slot = (crank + CS - q - 1) % CS;      // this CTA's place in q's buffer
+                const uint32_t dst = mapa_cluster(x_base + (slot * TC_BM + (uint32_t)r) * (uint32_t)(W * 4), q);
+                const uint32_t src = taddr + q * (uint32_t)W;
+                tmem_ld16_issue(src, ra);
+                for (int c = 0; c < W; c += 32) {
+                    tmem_ld_wait16(ra);
+                    tmem_ld16_issue(src + (uint32_t)(c + 16), rb);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v)
+                        st_cluster_v4(dst + ((((uint32_t)(c >> 2) + v) ^ swz) << 4), ra[4 * v], ra[4 * v + 1], ra[4 * v + 2], ra[4 * v + 3]);
+                    tmem_ld_wait16(rb);
+                    if (c + 32 < W) tmem_ld16_issue(src + (uint32_t)(c + 32), ra);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v)
+                        st_cluster_v4(dst + ((((uint32_t)(c >> 2) + 4 + v) ^ swz) << 4), rb[4 * v], rb[4 * v + 1], rb[4 * v + 2], rb[4 * v + 3]);
+                }
+                fence_cluster();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_release_cluster(mapa_cluster(smem_u32(&sh.x_full), q));
+            }
+            // ---- reduce: own centroid range, own partials plus the peers'
+            if (!mbar_wait_cluster_warp(smem_u32(&sh.x_full), ti & 1u, abort_flag, p.ctl)) { ok = false; break; }
+            float b1 = TC_KEY_INIT, b2 = TC_KEY_INIT, b3 = TC_KEY_INIT, b4 = TC_KEY_INIT;
+            {
+                const int k0 = (int)crank * W;
+                const uint32_t src = taddr + (uint32_t)k0;
+                tmem_ld16_issue(src, ra);
+                for (int c = 0; c < W; c += 16) {
+                    tmem_ld_wait16(ra);
+                    float acc[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(ra[j]);
+                    if (c + 16 < W) tmem_ld16_issue(src + (uint32_t)(c + 16), ra);
+#pragma unroll
+                    for (int slot = 0; slot < CS - 1; ++slot) {
+                        const unsigned char *xr = x_ptr + ((size_t)slot * TC_BM + r) * (size_t)(W * 4);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            const float4 t = *reinterpret_cast<const float4 *>(xr + ((((uint32_t)(c >> 2) + v) ^ swz) << 4));
+                            acc[4 * v] += t.x;
+                            acc[4 * v + 1] += t.y;
+                            acc[4 * v + 2] += t.z;
+                            acc[4 * v + 3] += t.w;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        key_insert(make_key(fmaf(-2.f, acc[j], sh.cn[k0 + c + j]), k0 + c + j), b1, b2, b3, b4);
+                }
+            }
+            if (quarter == 0 && lane == 0) TC_TRACE(ti, 5);
+            // accumulator buffer b and the exchange buffer are free from here on
+            tc_fence_before();
+            fence_cluster();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&sh.tmem_empty[b]));
+#pragma unroll 1
+                for (uint32_t d = 1; d < (uint32_t)CS; ++d)
+                    mbar_arrive_release_cluster(mapa_cluster(smem_u32(&sh.x_empty), (crank + d) % CS));
+            }
+            // ---- the four smallest keys of a row go to its owner, which merges the CS lists
+            if (owner != crank) {
+                const uint32_t dst = mapa_cluster(smem_u32(&sh.peer_key[b][crank * RP + (uint32_t)(r - (int)owner * RP)]), owner);
+                st_cluster_v4(dst, __float_as_uint(b1), __float_as_uint(b2), __float_as_uint(b3), __float_as_uint(b4));
+                fence_cluster();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_release_cluster(mapa_cluster(smem_u32(&sh.k_full[b]), owner));
+            } else {
+                if (!mbar_wait_cluster_warp(smem_u32(&sh.k_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
+                const int rl = r - (int)crank * RP;
+#pragma unroll
+                for (int d = 1; d < CS; ++d) {
+                    const float4 t = sh.peer_key[b][((crank + d) % CS) * RP + rl];
+                    key_insert(t.x, b1, b2, b3, b4);
+                    key_insert(t.y, b1, b2, b3, b4);
+                    key_insert(t.z, b1, b2, b3, b4);
+                    key_insert(t.w, b1, b2, b3, b4);
+                }
+                if (!mbar_wait_warp(smem_u32(&sh.lab_empty[b]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                sh.top_key[b][rl] = make_float4(b1, b2, b3, b4);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.lab_full[b]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ streaming warps
+        setmaxnreg_inc<TC_REGS_STREAM>();
+        const int ew = warp - TC_FIRST_STREAM_WARP;
+        uint32_t ti = 0;
+        bool ok = true;
+        for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
+            const int b = ti & 1;
+            const uint32_t ph = (ti >> 1) & 1u;
+            const int64_t row0 = unit * TC_BM + (int64_t)crank * RP;
+            if (!mbar_wait_warp(smem_u32(&sh.lab_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
+            if (ew == 0 && lane == 0) TC_TRACE(ti, 6);
+            for (int rl = ew; rl < RP; rl += TC_STREAM_WARPS) {
+                const int64_t row = row0 + rl;
+                if (row < p.N) stream_row(p, row, sh.top_key[b][rl], cmax2, lane);
+                __syncwarp();
+                if (lane == 0) atomicAdd(&sh.rows_streamed, 1);
+            }
+            __syncwarp();
+            if (ew == 0 && lane == 0) TC_TRACE(ti, 7);
+            if (lane == 0) mbar_arrive(smem_u32(&sh.lab_empty[b]));
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();   // no CTA's shared memory goes away while a peer may still write to it
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
 // Squared row norms (labels-only mode), slightly over-estimated to keep the error bound on the safe
 // side; with amax_bits also the largest magnitude of the matrix (as the bits of a non-negative float,
 // which order like unsigned integers).  A row is read by G lanes, G = the power of two >= D / 4
@@ -1177,6 +1560,98 @@ cudaError_t launch_wait_selftest(Control *ctl, int limit_ms, cudaStream_t s)
     return cudaGetLastError();
 }
 
+// ---- column-split inference kernel: selection and launch
+static std::atomic<int> g_apply_split{0};   // 0 = chosen here, 1 = never, 2 / 4 = that cluster size where it applies
+
+void set_apply_column_split(int cs) { g_apply_split.store((cs == 1 || cs == 2 || cs == 4) ? cs : 0, std::memory_order_relaxed); }
+int get_apply_column_split() { return g_apply_split.load(std::memory_order_relaxed); }
+
+namespace {
+
+struct SplitGeometry {
+    int npad, a_stages, b_stages;
+    size_t smem;
+};
+
+// false if a cluster of cs CTAs cannot take this shape
+bool split_geometry(int cs, int64_t N, int D, int K, SplitGeometry *g)
+{
+    if (N <= TC_BM || D < 128 || D % (32 * cs) != 0) return false;
+    const int unit = 32 * cs;
+    g->npad = (K + unit - 1) / unit * unit;
+    if (g->npad > 256) return false;
+    g->b_stages = TC_AFFINE_B_STAGES;
+    const size_t b_bytes = (size_t)g->npad * 128;
+    const size_t x_bytes = (size_t)(cs - 1) * TC_BM * (g->npad / cs) * 4;
+    const size_t fixed = 1024 + g->b_stages * b_bytes + x_bytes + sizeof(TcSplitShared);
+    const size_t budget = 227 * 1024;
+    if (fixed + 2 * TC_A_BYTES > budget) return false;
+    int a = (int)((budget - fixed) / TC_A_BYTES);
+    if (a > TC_AFFINE_A_STAGES) a = TC_AFFINE_A_STAGES;
+    g->a_stages = a;
+    g->smem = fixed + (size_t)a * TC_A_BYTES;
+    return true;
+}
+
+int choose_column_split(int64_t N, int D, int K)
+{
+    const int mode = g_apply_split.load(std::memory_order_relaxed);
+    if (mode == 1) return 1;
+    SplitGeometry g;
+    if (mode > 1) return split_geometry(mode, N, D, K, &g) ? mode : 1;
+    return 1;
+}
+
+cudaError_t launch_apply_split(int cs, TcParams p, const float *C, cudaStream_t s)
+{
+    SplitGeometry g;
+    if (!split_geometry(cs, p.N, p.D, p.K, &g)) return cudaErrorInvalidValue;
+    p.npad = g.npad;
+    int cols = 32;
+    while (cols < 2 * p.npad) cols <<= 1;
+    p.tmem_cols = cols;
+    p.a_stages = g.a_stages;
+    p.b_stages = g.b_stages;
+    CUtensorMap mapA, mapB;
+    if (!make_map(&mapA, p.Y, false, p.N, p.D, TC_BM) || !make_map(&mapB, C, false, p.K, p.D, p.npad))
+        return cudaErrorInvalidValue;
+    const void *kern = cs == 2 ? reinterpret_cast<const void *>(apply_split_kernel<2>)
+                               : reinterpret_cast<const void *>(apply_split_kernel<4>);
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem)) != cudaSuccess) return e;
+    if (!regs_ok(kern)) return cudaErrorLaunchOutOfResources;
+
+    cudaLaunchConfig_t cfg{};
+    cfg.blockDim = dim3(TC_THREADS_AFFINE, 1, 1);
+    cfg.dynamicSmemBytes = g.smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // one resident cluster per cs SMs, as many as the device can hold at once
+    int64_t clusters = sm_count() / cs;
+    {
+        cfg.gridDim = dim3((unsigned)(clusters * cs), 1, 1);
+        int resident = 0;
+        if (cudaOccupancyMaxActiveClusters(&resident, kern, &cfg) == cudaSuccess && resident > 0 && resident < clusters)
+            clusters = resident;
+    }
+    const int64_t units = (p.N + TC_BM - 1) / TC_BM;
+    if (units < clusters) clusters = units;
+    cfg.gridDim = dim3((unsigned)(clusters * cs), 1, 1);
+    if (cs == 2) e = cudaLaunchKernelEx(&cfg, apply_split_kernel<2>, mapA, mapB, p);
+    else e = cudaLaunchKernelEx(&cfg, apply_split_kernel<4>, mapA, mapB, p);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
 bool tc_half_supported(int64_t N, int D, int K)
 {
     return tc_supported(N, D, K) && (D % 8 == 0);
@@ -1211,6 +1686,10 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     const bool affine = out != nullptr;
     const bool half = (Yh != nullptr) && !affine;
     p.scale = scale;
+    if (affine) {
+        const int cs = choose_column_split(N, D, K);
+        if (cs > 1) return launch_apply_split(cs, p, C, s);
+    }
     // Two CTAs per 256 rows whenever there is more than one tile of rows.
     const bool pair = N > TC_BM;
     const int nb_rows = pair ? p.npad / 2 : p.npad;

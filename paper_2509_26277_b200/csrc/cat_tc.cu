@@ -341,9 +341,13 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, uint32_t fmt)
 constexpr int TC_TRACE_TILES = 16;
 constexpr int TC_TRACE_EVENTS = 8;
 __device__ unsigned long long g_tc_trace[2][TC_TRACE_TILES][TC_TRACE_EVENTS];
+#ifndef CAT_TC_TRACE_FIRST
+#define CAT_TC_TRACE_FIRST 0
+#endif
 #define TC_TRACE(ti, ev)                                                                               \
     do {                                                                                               \
-        if (blockIdx.x < 2 && (ti) < TC_TRACE_TILES) g_tc_trace[blockIdx.x][ti][ev] = global_timer();  \
+        if (blockIdx.x < 2 && (ti) >= CAT_TC_TRACE_FIRST && (ti) < CAT_TC_TRACE_FIRST + TC_TRACE_TILES) \
+            g_tc_trace[blockIdx.x][(ti) - CAT_TC_TRACE_FIRST][ev] = global_timer();                    \
     } while (0)
 #else
 #define TC_TRACE(ti, ev) do { } while (0)
@@ -898,6 +902,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 // those, and sends them to the CTA that owns the row (rows [q 128 / CS, (q + 1) 128 / CS) belong
 // to CTA q), which merges the CS lists and streams the row out.  Per CTA only 128 / CS rows'
 // worth of bytes is in flight; the price is CS times the centroid bytes out of L2 per row.
+// Its streaming warps get by with two warpgroups (the bytes in flight per SM are what counts, and a
+// row keeps 24 float4 per lane in flight either way), which leaves each of them 208 registers:
+// with three warpgroups of 128 the exchange code pushed the streaming loop into spills.
+constexpr int TCS_STREAM_WARPS = 8;
+constexpr int TCS_THREADS = 32 * (TC_FIRST_STREAM_WARP + TCS_STREAM_WARPS);   // 512
+constexpr int TCS_REGS_LAUNCH = 128;
+constexpr int TCS_REGS_STREAM = 208;
+static_assert(128 * (TC_REGS_CONTROL + TC_REGS_SCORE + (TCS_STREAM_WARPS / 4) * TCS_REGS_STREAM) <= TCS_REGS_LAUNCH * TCS_THREADS,
+              "register split exceeds what the block is launched with");
+
 struct TcSplitShared {
     uint64_t a_full[TC_MAX_A_STAGES];
     uint64_t a_empty[TC_MAX_A_STAGES];
@@ -966,7 +980,7 @@ __device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t pa
 }
 
 template <int CS>
-__global__ void __launch_bounds__(TC_THREADS_AFFINE, 1)
+__global__ void __launch_bounds__(TCS_THREADS, 1)
 apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p)
 {
     constexpr int RP = TC_BM / CS;                 // rows of a tile this CTA owns
@@ -1006,7 +1020,7 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             mbar_init(smem_u32(&sh.tmem_full[b]), 1);
             mbar_init(smem_u32(&sh.tmem_empty[b]), TC_SCORE_WARPS);
             mbar_init(smem_u32(&sh.lab_full[b]), OWNER_WARPS);
-            mbar_init(smem_u32(&sh.lab_empty[b]), TC_STREAM_WARPS);
+            mbar_init(smem_u32(&sh.lab_empty[b]), TCS_STREAM_WARPS);
             mbar_init(smem_u32(&sh.k_full[b]), (CS - 1) * OWNER_WARPS);
         }
         mbar_init(smem_u32(&sh.x_full), (CS - 1) * TC_SCORE_WARPS);
@@ -1051,7 +1065,7 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     const int row0 = (int)(unit * TC_BM);
                     if (ti > 1) {
                         // at most one tile ahead of the streaming warps
-                        if (!wait_progress(&sh.rows_streamed, (int)(ti - 1) * RP, abort_flag, p.ctl)) { ok = false; break; }
+                        if (!wait_progress(&sh.rows_streamed, (int)(ti - 1) * RP - RP / 2, abort_flag, p.ctl)) { ok = false; break; }
                     }
                     for (int sl = 0; sl < nslabs; ++sl) {
                         if (!mbar_wait(smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
@@ -1163,7 +1177,7 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     for (int v = 0; v < 4; ++v)
                         st_cluster_v4(dst + ((((uint32_t)(c >> 2) + 4 + v) ^ swz) << 4), rb[4 * v], rb[4 * v + 1], rb[4 * v + 2], rb[4 * v + 3]);
                 }
-                fence_cluster();
+                // (no separate fence: __syncwarp orders the lanes, the arrival below releases at cluster scope)
                 __syncwarp();
                 if (lane == 0) mbar_arrive_release_cluster(mapa_cluster(smem_u32(&sh.x_full), q));
             }
@@ -1173,13 +1187,13 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             {
                 const int k0 = (int)crank * W;
                 const uint32_t src = taddr + (uint32_t)k0;
-                tmem_ld16_issue(src, ra);
+#pragma unroll 1
                 for (int c = 0; c < W; c += 16) {
-                    tmem_ld_wait16(ra);
+                    tmem_ld16_issue(src + (uint32_t)c, ra);
+                    // the peers' partials of these 16 centroids, read while the TMEM load is in flight
                     float acc[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(ra[j]);
-                    if (c + 16 < W) tmem_ld16_issue(src + (uint32_t)(c + 16), ra);
+                    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
 #pragma unroll
                     for (int slot = 0; slot < CS - 1; ++slot) {
                         const unsigned char *xr = x_ptr + ((size_t)slot * TC_BM + r) * (size_t)(W * 4);
@@ -1192,15 +1206,16 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                             acc[4 * v + 3] += t.w;
                         }
                     }
+                    tmem_ld_wait16(ra);
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        key_insert(make_key(fmaf(-2.f, acc[j], sh.cn[k0 + c + j]), k0 + c + j), b1, b2, b3, b4);
+                        key_insert(make_key(fmaf(-2.f, acc[j] + __uint_as_float(ra[j]), sh.cn[k0 + c + j]), k0 + c + j), b1, b2, b3, b4);
                 }
             }
             if (quarter == 0 && lane == 0) TC_TRACE(ti, 5);
             // accumulator buffer b and the exchange buffer are free from here on
             tc_fence_before();
-            fence_cluster();
+            // (no separate fence: __syncwarp orders the lanes, the arrival below releases at cluster scope)
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(smem_u32(&sh.tmem_empty[b]));
@@ -1212,7 +1227,7 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             if (owner != crank) {
                 const uint32_t dst = mapa_cluster(smem_u32(&sh.peer_key[b][crank * RP + (uint32_t)(r - (int)owner * RP)]), owner);
                 st_cluster_v4(dst, __float_as_uint(b1), __float_as_uint(b2), __float_as_uint(b3), __float_as_uint(b4));
-                fence_cluster();
+                // (no separate fence: __syncwarp orders the lanes, the arrival below releases at cluster scope)
                 __syncwarp();
                 if (lane == 0) mbar_arrive_release_cluster(mapa_cluster(smem_u32(&sh.k_full[b]), owner));
             } else {
@@ -1234,7 +1249,7 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         }
     } else {
         // ------------------------------------------------------------ streaming warps
-        setmaxnreg_inc<TC_REGS_STREAM>();
+        setmaxnreg_inc<TCS_REGS_STREAM>();
         const int ew = warp - TC_FIRST_STREAM_WARP;
         uint32_t ti = 0;
         bool ok = true;
@@ -1244,7 +1259,7 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             const int64_t row0 = unit * TC_BM + (int64_t)crank * RP;
             if (!mbar_wait_warp(smem_u32(&sh.lab_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
             if (ew == 0 && lane == 0) TC_TRACE(ti, 6);
-            for (int rl = ew; rl < RP; rl += TC_STREAM_WARPS) {
+            for (int rl = ew; rl < RP; rl += TCS_STREAM_WARPS) {
                 const int64_t row = row0 + rl;
                 if (row < p.N) stream_row(p, row, sh.top_key[b][rl], cmax2, lane);
                 __syncwarp();
@@ -1588,6 +1603,9 @@ bool split_geometry(int cs, int64_t N, int D, int K, SplitGeometry *g)
     if (fixed + 2 * TC_A_BYTES > budget) return false;
     int a = (int)((budget - fixed) / TC_A_BYTES);
     if (a > TC_AFFINE_A_STAGES) a = TC_AFFINE_A_STAGES;
+    // the streaming warps need the L1 that a carve-out above 196 KB takes away: give up a stage for it
+    const size_t soft = 195 * 1024;
+    while (a > 2 && fixed + (size_t)a * TC_A_BYTES > soft) --a;
     g->a_stages = a;
     g->smem = fixed + (size_t)a * TC_A_BYTES;
     return true;
@@ -1619,10 +1637,15 @@ cudaError_t launch_apply_split(int cs, TcParams p, const float *C, cudaStream_t 
                                : reinterpret_cast<const void *>(apply_split_kernel<4>);
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem)) != cudaSuccess) return e;
-    if (!regs_ok(kern)) return cudaErrorLaunchOutOfResources;
+    {
+        cudaFuncAttributes fa{};
+        if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return cudaErrorInvalidValue;
+        if ((long)fa.numRegs * TCS_THREADS < 128L * (TC_REGS_CONTROL + TC_REGS_SCORE + (TCS_STREAM_WARPS / 4) * TCS_REGS_STREAM))
+            return cudaErrorLaunchOutOfResources;
+    }
 
     cudaLaunchConfig_t cfg{};
-    cfg.blockDim = dim3(TC_THREADS_AFFINE, 1, 1);
+    cfg.blockDim = dim3(TCS_THREADS, 1, 1);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];

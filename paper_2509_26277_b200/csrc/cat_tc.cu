@@ -664,8 +664,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 bool ok = true;
                 for (int64_t unit = unit_first; unit < num_units && ok; unit += unit_step, ++ti) {
                     const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
-                    if (AFFINE && ti > 1) {
+                    if (AFFINE && !SHORT && ti > 1) {
                         // at most one tile ahead of the streaming warps: tile ti - 2 is streamed out
+                        // (short rows: a tile is a few KB, the ring depths alone bound the lead)
                         if (!wait_progress(&sh.rows_streamed, (int)(ti - 1) * TC_BM, abort_flag, p.ctl)) { ok = false; break; }
                     }
                     for (int sl = 0; sl < nslabs; ++sl) {
@@ -799,12 +800,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             const int b = ti & 1;
             const uint32_t ph = (ti >> 1) & 1u;
             const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
+            // what the certainty test needs from global memory is requested before the wait for the
+            // scores, so that its latency passes during the MMAs (fp16 operands: this thread's row has
+            // its own scale)
+            float rinv = 1.f, yn2 = 0.f;
+            if (HALF && row0 + quarter * 32 + lane < p.N) rinv = p.scale[4 + row0 + quarter * 32 + lane];
+            if (!AFFINE && row0 + quarter * 32 + lane < p.N) yn2 = p.ynorm2[row0 + quarter * 32 + lane];
             if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
             tc_fence_after();
             if (quarter == 0 && lane == 0) TC_TRACE(ti, 4);
-            // fp16 operands: this thread's row has its own scale
-            float rinv = 1.f;
-            if (HALF && row0 + quarter * 32 + lane < p.N) rinv = p.scale[4 + row0 + quarter * 32 + lane];
             const float coef = coef_c * rinv;
             float b1 = TC_KEY_INIT, b2 = TC_KEY_INIT, b3 = TC_KEY_INIT, b4 = TC_KEY_INIT;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
@@ -841,8 +845,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             } else {
                 const int64_t row = row0 + r;
                 if (row < p.N) {
-                    const float e = HALF ? tc_error_bound_half(p.D, p.ynorm2[row], cmax2, 2.9802322e-8f * rinv, abs_err_c)
-                                         : tc_error_bound(p.D, p.ynorm2[row], cmax2);
+                    const float e = HALF ? tc_error_bound_half(p.D, yn2, cmax2, 2.9802322e-8f * rinv, abs_err_c)
+                                         : tc_error_bound(p.D, yn2, cmax2);
                     p.labels[row] = key_label(b1, p.K);
                     tc_decide(p, row, make_float4(b1, b2, b3, b4), e);
                 }

@@ -36,6 +36,28 @@ def test_version_and_status_strings():
     assert L.cat_status_string(99) == b"unknown status"
 
 
+def test_kernel_selection_settings_are_host_state():
+    """Both selectors are process-wide host settings: readable and writable without a GPU."""
+    assert binding.cat_get_apply_column_split() == 0
+    try:
+        for cs in (1, 2, 4):
+            binding.cat_set_apply_column_split(cs)
+            assert binding.cat_get_apply_column_split() == cs
+        for bad in (3, 8, -1, 100):
+            binding.cat_set_apply_column_split(bad)
+            assert binding.cat_get_apply_column_split() == 0
+    finally:
+        binding.cat_set_apply_column_split(0)
+    k = binding.cat_get_tensor_core_min_k()
+    try:
+        binding.cat_set_tensor_core_min_k(64)
+        assert binding.cat_get_tensor_core_min_k() == 64
+        binding.cat_set_tensor_core_min_k(0)
+        assert binding.cat_get_tensor_core_min_k() == 1
+    finally:
+        binding.cat_set_tensor_core_min_k(k)
+
+
 def test_workspace_queries_are_pure_host_functions():
     L = binding.lib()
     a = L.cat_apply_workspace_bytes(50_000, 1000, 16)

@@ -198,6 +198,52 @@ def test_tensor_paths_shapes_and_scales(n, d, k, scale):
     close(host(out) / scale, want2 / scale, "outputs")
 
 
+@pytest.mark.parametrize("cs", [2, 4])
+@pytest.mark.parametrize("n,d,k", [(3000, 256, 48), (1111, 1024, 256), (700, 128, 32), (2500, 512, 200),
+                                   (129, 128, 33), (40000, 256, 64)])
+def test_apply_column_split_matches_oracle(n, d, k, cs):
+    """The column-split form of the fused inference kernel (clusters of 2 or 4 CTAs share a 128-row
+    tile and sum partial scores through distributed shared memory): ragged N, K that does not fill
+    the cluster's centroid ranges, several tiles per cluster.  Same bar as the row-tile form, and
+    bit-identical outputs to it."""
+    rng = np.random.default_rng(n + d + k)
+    cen = (rng.normal(size=(k, d)) * 2).astype(np.float32)
+    Yq = (cen[rng.integers(0, k, size=n)] + rng.normal(size=(n, d))).astype(np.float32)
+    C = (cen + 0.05 * rng.normal(size=cen.shape)).astype(np.float32)
+    G = rng.normal(size=(k, d)).astype(np.float32)
+    Bt = rng.normal(size=(k, d)).astype(np.float32)
+    want, lab, best, second = O.apply(Yq, C, G, Bt)
+    assert B.cat_get_apply_column_split() == 0
+    try:
+        B.cat_set_apply_column_split(1)
+        ref, _ = B.cat_apply(dev(Yq), dev(C), dev(G), dev(Bt), want_labels=True)
+        B.cat_set_apply_column_split(cs)
+        ws = B.workspace("apply", n, d, k, "cuda")
+        out, glab = B.cat_apply(dev(Yq), dev(C), dev(G), dev(Bt), want_labels=True, ws=ws)
+        rep = B.cat_workspace_report(ws)
+    finally:
+        B.cat_set_apply_column_split(0)
+    assert rep["device_status"] == 0
+    _, n_diff = labels_match(host(glab), lab, best, second, "apply labels (column split)")
+    want2 = want if n_diff == 0 else O.affine_with_labels(Yq, host(glab), G, Bt)
+    close(host(out), want2, "outputs (column split)")
+    assert torch.equal(out, ref)
+
+
+def test_apply_column_split_falls_back_where_the_shape_does_not_allow_it():
+    """D not a multiple of 32 cs: the request is ignored and the row-tile kernel runs."""
+    w, _ = workload("cfg2")
+    C, G, Bt, _ = B.cat_fit(dev(w.Yq_fit.numpy()), dev(w.Yfp_fit.numpy()), w.K, 3)
+    Y = dev(w.Yq_apply.numpy()[:5000])
+    ref = B.cat_apply(Y, C, G, Bt)
+    try:
+        B.cat_set_apply_column_split(4)
+        out = B.cat_apply(Y, C, G, Bt)
+    finally:
+        B.cat_set_apply_column_split(0)
+    assert torch.equal(out, ref)
+
+
 def test_fit_fp16_and_tf32_operands_agree():
     """The default start lets cat_fit assign from an fp16 copy of the rows; an explicit start (here the
     same first K rows) keeps TF32 operands.  Labels are decided exactly either way."""

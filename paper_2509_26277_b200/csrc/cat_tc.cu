@@ -515,6 +515,51 @@ __device__ __forceinline__ void stream_row(const TcParams &p, int64_t row, float
     }
 }
 
+// Streaming of one row without the certainty test: out = gamma_l * y + beta_l, returns ||y||^2
+// (complete in every lane).  The column-split kernel decides certainty in its score warps, which
+// leaves the streaming loop the registers for 24 loads per lane in flight and little else.
+__device__ __forceinline__ float stream_row_lean(const TcParams &p, int64_t row, int l, int lane)
+{
+    const int D4 = p.D >> 2;
+    const float4 *y4 = reinterpret_cast<const float4 *>(p.Y) + (size_t)row * D4 + lane;
+    const float4 *g4 = reinterpret_cast<const float4 *>(p.gamma) + (size_t)l * D4 + lane;
+    const float4 *b4 = reinterpret_cast<const float4 *>(p.beta) + (size_t)l * D4 + lane;
+    float4 *o4 = reinterpret_cast<float4 *>(p.out) + (size_t)row * D4 + lane;
+    float ysq = 0.f;
+#pragma unroll 1
+    for (int h = 0; h < D4; h += 256) {
+        float4 y[8], g[8], bb[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int c = h + 32 * q;
+            if (c + lane < D4) {
+                y[q] = __ldcs(y4 + c);
+                g[q] = __ldg(g4 + c);
+                bb[q] = __ldg(b4 + c);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int c = h + 32 * q;
+            if (c + lane < D4) {
+                float4 v;
+                v.x = fmaf(g[q].x, y[q].x, bb[q].x);
+                v.y = fmaf(g[q].y, y[q].y, bb[q].y);
+                v.z = fmaf(g[q].z, y[q].z, bb[q].z);
+                v.w = fmaf(g[q].w, y[q].w, bb[q].w);
+                __stcs(o4 + c, v);
+                ysq = fmaf(y[q].x, y[q].x, ysq);
+                ysq = fmaf(y[q].y, y[q].y, ysq);
+                ysq = fmaf(y[q].z, y[q].z, ysq);
+                ysq = fmaf(y[q].w, y[q].w, ysq);
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
+    return ysq;
+}
+
 // The same for short rows (D < 128): a row takes only G = 1 .. 16 lanes, so a warp streams all
 // of its rows of the tile (ew, ew + TC_STREAM_WARPS, ...) in one step, 32 / G rows per load slot.
 __device__ __forceinline__ void stream_rows_short(const TcParams &p, int64_t row0, const float4 *tile_keys, int ew,
@@ -906,13 +951,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
 // those, and sends them to the CTA that owns the row (rows [q 128 / CS, (q + 1) 128 / CS) belong
 // to CTA q), which merges the CS lists and streams the row out.  Per CTA only 128 / CS rows'
 // worth of bytes is in flight; the price is CS times the centroid bytes out of L2 per row.
-// Its streaming warps get by with two warpgroups (the bytes in flight per SM are what counts, and a
-// row keeps 24 float4 per lane in flight either way), which leaves each of them 208 registers:
-// with three warpgroups of 128 the exchange code pushed the streaming loop into spills.
-constexpr int TCS_STREAM_WARPS = 8;
-constexpr int TCS_THREADS = 32 * (TC_FIRST_STREAM_WARP + TCS_STREAM_WARPS);   // 512
-constexpr int TCS_REGS_LAUNCH = 128;
-constexpr int TCS_REGS_STREAM = 208;
+// Its warp roles and register split are those of the row-tile kernel (three streaming warpgroups of
+// 128 registers).  The streaming loop holds 24 float4 per lane in flight, which leaves 32 registers
+// for everything else: the certainty test therefore runs in the score warps (one thread per row,
+// from the row norms the streaming warps leave in shared memory), not in the streaming loop.  With
+// the test inside the loop the compiler spilled there, and a spill in that loop doubles the
+// kernel's run time.
+constexpr int TCS_STREAM_WARPS = 12;
+constexpr int TCS_THREADS = 32 * (TC_FIRST_STREAM_WARP + TCS_STREAM_WARPS);   // 640
+constexpr int TCS_REGS_LAUNCH = 96;
+constexpr int TCS_REGS_STREAM = 128;
 static_assert(128 * (TC_REGS_CONTROL + TC_REGS_SCORE + (TCS_STREAM_WARPS / 4) * TCS_REGS_STREAM) <= TCS_REGS_LAUNCH * TCS_THREADS,
               "register split exceeds what the block is launched with");
 
@@ -936,6 +984,7 @@ struct TcSplitShared {
     float cn[256];
     float4 top_key[2][TC_BM];     // merged keys of the rows this CTA owns (the first 128 / CS entries)
     float4 peer_key[2][TC_BM];    // [buffer][source CTA * (128 / CS) + row]
+    float row_norm[2][TC_BM];     // ||y||^2 of the rows this CTA streamed, by the streaming warps
 };
 
 __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
@@ -1246,9 +1295,32 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     key_insert(t.w, b1, b2, b3, b4);
                 }
                 if (!mbar_wait_warp(smem_u32(&sh.lab_empty[b]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
+                if (ti >= 2) {
+                    // tile ti - 2 (same buffer) is streamed out: its row norms are in, its keys still here
+                    const int64_t row = (unit - 2 * unit_step) * TC_BM + (int64_t)crank * RP + rl;
+                    if (row < p.N) {
+                        const float4 keys = sh.top_key[b][rl];
+                        p.labels[row] = key_label(keys.x, p.K);
+                        tc_decide(p, row, keys, tc_error_bound(p.D, sh.row_norm[b][rl] * 1.0001f, cmax2));
+                    }
+                }
                 sh.top_key[b][rl] = make_float4(b1, b2, b3, b4);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&sh.lab_full[b]));
+            }
+        }
+        // the last two tiles are decided once the streaming warps are through with them
+        if (ok && owner == crank) {
+            const int rl = r - (int)crank * RP;
+            for (uint32_t t = (ti >= 2 ? ti - 2 : 0); t < ti; ++t) {
+                const int b = t & 1;
+                if (!mbar_wait_warp(smem_u32(&sh.lab_empty[b]), (t >> 1) & 1u, abort_flag, p.ctl)) break;
+                const int64_t row = (unit_first + (int64_t)t * unit_step) * TC_BM + (int64_t)crank * RP + rl;
+                if (row < p.N) {
+                    const float4 keys = sh.top_key[b][rl];
+                    p.labels[row] = key_label(keys.x, p.K);
+                    tc_decide(p, row, keys, tc_error_bound(p.D, sh.row_norm[b][rl] * 1.0001f, cmax2));
+                }
             }
         }
     } else {
@@ -1265,7 +1337,10 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             if (ew == 0 && lane == 0) TC_TRACE(ti, 6);
             for (int rl = ew; rl < RP; rl += TCS_STREAM_WARPS) {
                 const int64_t row = row0 + rl;
-                if (row < p.N) stream_row(p, row, sh.top_key[b][rl], cmax2, lane);
+                if (row < p.N) {
+                    const float ysq = stream_row_lean(p, row, key_label(sh.top_key[b][rl].x, p.K), lane);
+                    if (lane == 0) sh.row_norm[b][rl] = ysq;
+                }
                 __syncwarp();
                 if (lane == 0) atomicAdd(&sh.rows_streamed, 1);
             }

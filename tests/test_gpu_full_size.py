@@ -87,4 +87,14 @@ def test_config4_full_size():
         y = w.Yq_apply[sl][:, cols].double()
         ref = (G[l][:, cols].double() * y + Bt[l][:, cols].double()).float()
         assert torch.equal(ref, out[sl][:, cols])
+    # the column-split form of the kernel gives the same labels and the same bits
+    del y, ref, l
+    try:
+        B.cat_set_apply_column_split(2)
+        out2, alab2 = B.cat_apply(w.Yq_apply, C, G, Bt, want_labels=True)
+        torch.cuda.synchronize()
+    finally:
+        B.cat_set_apply_column_split(0)
+    assert torch.equal(alab2, alab)
+    assert torch.equal(out2, out)
     B.clear_workspaces()

@@ -532,6 +532,9 @@ __global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
     if ((int64_t)count > N) count = (int)N;
     if (blockIdx.x == 0 && threadIdx.x == 0) ctl->refined_total += count;
     const int lane = threadIdx.x & 31;
+    const bool vec4 = (D & 3) == 0 && ((reinterpret_cast<uintptr_t>(Y) | reinterpret_cast<uintptr_t>(C)) & 15u) == 0 &&
+                      (!AFFINE || ((reinterpret_cast<uintptr_t>(gamma) | reinterpret_cast<uintptr_t>(beta) |
+                                    reinterpret_cast<uintptr_t>(out)) & 15u) == 0);
     const int gw = blockIdx.x * (RC_THREADS / 32) + (threadIdx.x >> 5);
     const int nw = gridDim.x * (RC_THREADS / 32);
     for (int it = gw; it < count; it += nw) {
@@ -550,7 +553,44 @@ __global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
         }
         const float *y = Y + (size_t)row * D;
         double s[4] = {0.0, 0.0, 0.0, 0.0};
-        if (ncand <= 2) {
+        if (vec4) {
+            // rows and centroids as 128-bit loads (D a multiple of 4, bases 16-byte aligned)
+            const float4 *y4 = reinterpret_cast<const float4 *>(y);
+            const int D4 = D >> 2;
+            if (ncand <= 2) {
+                const float4 *c0 = reinterpret_cast<const float4 *>(cp[0]);
+                const float4 *c1 = reinterpret_cast<const float4 *>(cp[1]);
+                // (unrolled so that the loads of several steps are in flight together: one warp walks
+                // its row alone, and a step that waited for its own loads cost a memory latency each)
+#pragma unroll 8
+                for (int j = lane; j < D4; j += 32) {
+                    const float4 yv = y4[j], a = c0[j], b = c1[j];
+                    double d;
+                    d = (double)yv.x - (double)a.x; s[0] = fma(d, d, s[0]);
+                    d = (double)yv.y - (double)a.y; s[0] = fma(d, d, s[0]);
+                    d = (double)yv.z - (double)a.z; s[0] = fma(d, d, s[0]);
+                    d = (double)yv.w - (double)a.w; s[0] = fma(d, d, s[0]);
+                    d = (double)yv.x - (double)b.x; s[1] = fma(d, d, s[1]);
+                    d = (double)yv.y - (double)b.y; s[1] = fma(d, d, s[1]);
+                    d = (double)yv.z - (double)b.z; s[1] = fma(d, d, s[1]);
+                    d = (double)yv.w - (double)b.w; s[1] = fma(d, d, s[1]);
+                }
+            } else {
+#pragma unroll 4
+                for (int j = lane; j < D4; j += 32) {
+                    const float4 yv = y4[j];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 c = reinterpret_cast<const float4 *>(cp[q])[j];
+                        double d;
+                        d = (double)yv.x - (double)c.x; s[q] = fma(d, d, s[q]);
+                        d = (double)yv.y - (double)c.y; s[q] = fma(d, d, s[q]);
+                        d = (double)yv.z - (double)c.z; s[q] = fma(d, d, s[q]);
+                        d = (double)yv.w - (double)c.w; s[q] = fma(d, d, s[q]);
+                    }
+                }
+            }
+        } else if (ncand <= 2) {
             // the common case: only the two nearest are in question
             for (int j = lane; j < D; j += 32) {
                 const double yv = (double)y[j];
@@ -589,7 +629,17 @@ __global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
             const float *g = gamma + (size_t)bk * D;
             const float *bb = beta + (size_t)bk * D;
             float *o = out + (size_t)row * D;
-            for (int j = lane; j < D; j += 32) o[j] = fmaf(g[j], y[j], bb[j]);
+            if (vec4) {
+                for (int j = lane; j < (D >> 2); j += 32) {
+                    const float4 yv = reinterpret_cast<const float4 *>(y)[j];
+                    const float4 gv = reinterpret_cast<const float4 *>(g)[j];
+                    const float4 bv = reinterpret_cast<const float4 *>(bb)[j];
+                    reinterpret_cast<float4 *>(o)[j] = make_float4(fmaf(gv.x, yv.x, bv.x), fmaf(gv.y, yv.y, bv.y),
+                                                                   fmaf(gv.z, yv.z, bv.z), fmaf(gv.w, yv.w, bv.w));
+                }
+            } else {
+                for (int j = lane; j < D; j += 32) o[j] = fmaf(g[j], y[j], bb[j]);
+            }
         }
     }
 }

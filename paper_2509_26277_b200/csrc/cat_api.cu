@@ -120,12 +120,12 @@ static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const fl
         if (Yh && !centroids_ready) CAT_CUDA(launch_to_half(C, (size_t)K * D, hscale, Ch, s));
         CAT_CUDA(launch_assign_tc(Y, N, D, K, C, w.cnorm, w.ynorm2, labels, w.refine_rows, w.cand_rows,
                                   w.cand_list, w.ctl, gamma, beta, out, s, Yh, Ch, hscale));
-        CAT_CUDA(launch_refine_candidates(Y, N, D, K, C, labels, w.cand_rows, w.cand_list, w.ctl, gamma,
-                                          beta, out, s));
+        CAT_CUDA(launch_refine_both(Y, N, D, K, C, labels, w.cand_rows, w.cand_list, w.refine_rows, w.ctl, gamma,
+                                    beta, out, s));
     } else {
         CAT_CUDA(launch_assign(Y, N, D, K, C, w.cnorm, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
+        if (K > 1) CAT_CUDA(launch_refine(Y, N, D, K, C, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
     }
-    if (K > 1) CAT_CUDA(launch_refine(Y, N, D, K, C, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
     return CAT_OK;
 }
 

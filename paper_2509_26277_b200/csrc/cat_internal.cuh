@@ -124,10 +124,9 @@ cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, 
 cudaError_t launch_to_half(const float *src, size_t n, const float *scale, void *dst, cudaStream_t s);
 
 // Exact fp64 decision among the listed candidates of each queued row; optional affine output.
-cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, const float *C,
-                                     int32_t *labels, const int32_t *cand_rows,
-                                     const uint64_t *cand_list, Control *ctl, const float *gamma,
-                                     const float *beta, float *out, cudaStream_t s);
+cudaError_t launch_refine_both(const float *Y, int64_t N, int D, int K, const float *C, int32_t *labels,
+                               const int32_t *cand_rows, const uint64_t *cand_list, const int32_t *refine_rows,
+                               Control *ctl, const float *gamma, const float *beta, float *out, cudaStream_t s);
 
 // Stable sort of the row indices by key.  prev == NULL (full mode): key = label, counts[k] = size of
 // cluster k.  prev != NULL (delta mode): entries only for rows with labels[i] != prev[i], under keys

@@ -423,12 +423,10 @@ constexpr int R_WARPS = R_THREADS / 32;
 // One CTA per queued row: warp w evaluates centroids w, w + 8, ... in direct form with fp64
 // accumulation; the CTA then takes the smallest distance, lowest index on equality.
 template <bool AFFINE>
-__global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restrict__ Y, int64_t N,
-                                                           int D, int K, const float *__restrict__ C,
-                                                           int32_t *labels,
-                                                           const int32_t *__restrict__ refine_rows,
-                                                           Control *ctl, const float *gamma,
-                                                           const float *beta, float *out)
+__device__ __forceinline__ void refine_body(const float *__restrict__ Y, int64_t N, int D, int K,
+                                            const float *__restrict__ C, int32_t *labels,
+                                            const int32_t *__restrict__ refine_rows, Control *ctl,
+                                            const float *gamma, const float *beta, float *out)
 {
     __shared__ double s_best[R_WARPS];
     __shared__ int s_idx[R_WARPS];
@@ -503,6 +501,17 @@ __global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restri
     }
 }
 
+template <bool AFFINE>
+__global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restrict__ Y, int64_t N,
+                                                           int D, int K, const float *__restrict__ C,
+                                                           int32_t *labels,
+                                                           const int32_t *__restrict__ refine_rows,
+                                                           Control *ctl, const float *gamma,
+                                                           const float *beta, float *out)
+{
+    refine_body<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out);
+}
+
 cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *C,
                           int32_t *labels, const int32_t *refine_rows, Control *ctl,
                           const float *gamma, const float *beta, float *out, cudaStream_t s)
@@ -523,7 +532,7 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
 constexpr int RC_THREADS = 256;
 
 template <bool AFFINE>
-__global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
+__device__ __forceinline__ void refine_candidates_body(
     const float *__restrict__ Y, int64_t N, int D, int K, const float *__restrict__ C, int32_t *labels,
     const int32_t *__restrict__ cand_rows, const uint64_t *__restrict__ cand_list, Control *ctl,
     const float *gamma, const float *beta, float *out, bool fast_output_valid)
@@ -644,19 +653,32 @@ __global__ void __launch_bounds__(RC_THREADS) refine_candidates_kernel(
     }
 }
 
-cudaError_t launch_refine_candidates(const float *Y, int64_t N, int D, int K, const float *C,
-                                     int32_t *labels, const int32_t *cand_rows,
-                                     const uint64_t *cand_list, Control *ctl, const float *gamma,
-                                     const float *beta, float *out, cudaStream_t s)
+// Both exact passes in one launch: the rows queued with their candidates (a warp each), then the
+// rows queued for a scan of all K (a CTA each).  A row is in one queue only.
+static_assert(RC_THREADS == R_THREADS, "the fused exact pass runs both bodies with one block size");
+template <bool AFFINE>
+__global__ void __launch_bounds__(R_THREADS) refine_both_kernel(
+    const float *__restrict__ Y, int64_t N, int D, int K, const float *__restrict__ C, int32_t *labels,
+    const int32_t *__restrict__ cand_rows, const uint64_t *__restrict__ cand_list,
+    const int32_t *__restrict__ refine_rows, Control *ctl, const float *gamma, const float *beta, float *out)
+{
+    refine_candidates_body<AFFINE>(Y, N, D, K, C, labels, cand_rows, cand_list, ctl, gamma, beta, out, AFFINE);
+    __syncthreads();   // (block 0's thread 0 updates the counters in both bodies, in this order)
+    refine_body<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out);
+}
+
+cudaError_t launch_refine_both(const float *Y, int64_t N, int D, int K, const float *C, int32_t *labels,
+                               const int32_t *cand_rows, const uint64_t *cand_list, const int32_t *refine_rows,
+                               Control *ctl, const float *gamma, const float *beta, float *out, cudaStream_t s)
 {
     int64_t want = (N + (RC_THREADS / 32) - 1) / (RC_THREADS / 32);
     int blocks = (int)(want < 1184 ? want : 1184);
     if (out)
-        refine_candidates_kernel<true><<<blocks, RC_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows,
-                                                                    cand_list, ctl, gamma, beta, out, true);
+        refine_both_kernel<true><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
+                                                             refine_rows, ctl, gamma, beta, out);
     else
-        refine_candidates_kernel<false><<<blocks, RC_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows,
-                                                                     cand_list, ctl, gamma, beta, out, false);
+        refine_both_kernel<false><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
+                                                              refine_rows, ctl, gamma, beta, out);
     count_launch();
     return cudaGetLastError();
 }

@@ -991,7 +991,6 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a,
 {
     asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
-__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 // arrival on a barrier of another CTA that publishes this thread's earlier (fenced) writes to it
 __device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_bar)
 {

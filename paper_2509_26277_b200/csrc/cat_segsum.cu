@@ -1,8 +1,8 @@
 // Segmented (per-cluster) sums through a stable sort of the rows by label.
 //
 //   label_hist_kernel     per-block key histograms (1024 entries per block)
-//   label_scan_blocks_kernel / label_scan_keys_kernel
-//                         per-block offsets, key totals, key offsets, segment table, cluster sizes
+//   label_scan_blocks_kernel  per-block offsets and key totals
+//                         (key offsets, segment table and cluster sizes: scan_keys, inside the scatter kernel)
 //   label_scatter_kernel  stable scatter of the row indices: order[] lists the rows of
 //                         key 0 in ascending row order, then key 1, ...
 //
@@ -128,17 +128,19 @@ __device__ __forceinline__ uint32_t cta_exclusive_scan(uint32_t v, uint32_t *wsu
 // settled clustering holds a handful): length = seg_rows_max * M / NE rounded up to 16, at least 16,
 // so that short lists still spread over many CTAs and the segment count stays within
 // NE / seg_rows_max + KK.
-__global__ void __launch_bounds__(1024) label_scan_keys_kernel(const uint32_t *__restrict__ key_total, int K, int KK,
-                                                                int seg_rows_max, int64_t NE, int delta,
-                                                                int64_t *__restrict__ counts,
-                                                                int32_t *__restrict__ cluster_start,
-                                                                int32_t *__restrict__ seg_start)
+// Runs in every CTA of the scatter kernel (each needs the key offsets for its own entries); the CTA
+// with `publish` set also writes the tables and updates the cluster sizes.  Returns this thread's
+// key offset (thread k < KK).
+__device__ __forceinline__ uint32_t scan_keys(const uint32_t *__restrict__ key_total, int K, int KK, int seg_rows_max,
+                                              int64_t NE, int delta, bool publish, int64_t *__restrict__ counts,
+                                              int32_t *__restrict__ cluster_start, int32_t *__restrict__ seg_start,
+                                              uint32_t *wsum /*[33] shared*/)
 {
-    __shared__ uint32_t wsum[33];
     const int k = threadIdx.x;
     const uint32_t tot = (k < KK) ? key_total[k] : 0u;
     uint32_t M = 0;
     const uint32_t ea = cta_exclusive_scan(tot, wsum, M);
+    if (!publish) return ea;
     int64_t sr = ((int64_t)seg_rows_max * (int64_t)M + NE - 1) / NE;
     sr = (sr + 15) / 16 * 16;
     if (sr < 16) sr = 16;
@@ -159,6 +161,7 @@ __global__ void __launch_bounds__(1024) label_scan_keys_kernel(const uint32_t *_
         if (delta) counts[k] += (int64_t)tot - (int64_t)key_total[K + k];
         else counts[k] = (int64_t)tot;
     }
+    return ea;
 }
 
 // Stable scatter.  Within a block, an entry's rank among the entries of its key is
@@ -166,12 +169,24 @@ __global__ void __launch_bounds__(1024) label_scan_keys_kernel(const uint32_t *_
 __global__ void __launch_bounds__(SORT_BLOCK) label_scatter_kernel(const int32_t *__restrict__ cur,
                                                                     const int32_t *__restrict__ prev, int64_t N, int K,
                                                                     int KK, const uint32_t *__restrict__ blk_hist,
-                                                                    const int32_t *__restrict__ cluster_start,
+                                                                    const uint32_t *__restrict__ key_total,
+                                                                    int seg_rows_max, int64_t NE, int delta,
+                                                                    int64_t *__restrict__ counts,
+                                                                    int32_t *__restrict__ cluster_start,
+                                                                    int32_t *__restrict__ seg_start,
                                                                     int32_t *__restrict__ order)
 {
-    extern __shared__ uint16_t warp_hist[];   // [32][KK]
+    extern __shared__ uint32_t scatter_smem[];   // [KK] key offsets, then [32][KK] 16-bit warp histograms
+    __shared__ uint32_t wsum[33];
+    uint32_t *key_off = scatter_smem;
+    uint16_t *warp_hist = reinterpret_cast<uint16_t *>(scatter_smem + KK);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     for (int e = tid; e < 32 * KK; e += SORT_BLOCK) warp_hist[e] = 0;
+    {
+        const uint32_t ea = scan_keys(key_total, K, KK, seg_rows_max, NE, delta, blockIdx.x == 0, counts, cluster_start,
+                                      seg_start, wsum);
+        if (tid < KK) key_off[tid] = ea;
+    }
     __syncthreads();
     const int64_t e = (int64_t)blockIdx.x * SORT_BLOCK + tid;
     const int l = entry_key(cur, prev, N, K, e);
@@ -189,7 +204,7 @@ __global__ void __launch_bounds__(SORT_BLOCK) label_scatter_kernel(const int32_t
     }
     __syncthreads();
     if (l >= 0) {
-        const uint32_t pos = (uint32_t)cluster_start[l] + blk_hist[(size_t)l * gridDim.x + blockIdx.x] +
+        const uint32_t pos = key_off[l] + blk_hist[(size_t)l * gridDim.x + blockIdx.x] +
                              warp_hist[w * KK + l] + (uint32_t)rank_in_warp;
         order[pos] = (int32_t)(e < N ? e : e - N);
     }
@@ -478,16 +493,18 @@ cudaError_t launch_label_sort(const int32_t *labels, const int32_t *prev, int64_
     const int KK = prev ? 2 * K : K;
     label_hist_kernel<<<g.nblk, SORT_BLOCK, (size_t)KK * sizeof(uint32_t), s>>>(labels, prev, N, K, KK, blk_hist);
     label_scan_blocks_kernel<<<(KK * 32 + 255) / 256, 256, 0, s>>>(blk_hist, g.nblk, KK, key_total);
-    label_scan_keys_kernel<<<1, 1024, 0, s>>>(key_total, K, KK, g.seg_rows, prev ? 2 * N : N, prev ? 1 : 0, counts,
-                                               cluster_start, seg_start);
-    const size_t sc_smem = (size_t)32 * KK * sizeof(uint16_t);
+    // (the scan over the keys -- key offsets, segment table, cluster sizes -- runs inside the scatter
+    // kernel: every CTA needs the offsets, CTA 0 publishes the tables)
+    const size_t sc_smem = (size_t)KK * sizeof(uint32_t) + (size_t)32 * KK * sizeof(uint16_t);
     if (sc_smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(label_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)sc_smem);
         if (e != cudaSuccess) return e;
     }
-    label_scatter_kernel<<<g.nblk, SORT_BLOCK, sc_smem, s>>>(labels, prev, N, K, KK, blk_hist, cluster_start, order);
-    count_launch(4);
+    label_scatter_kernel<<<g.nblk, SORT_BLOCK, sc_smem, s>>>(labels, prev, N, K, KK, blk_hist, key_total, g.seg_rows,
+                                                             prev ? 2 * N : N, prev ? 1 : 0, counts, cluster_start,
+                                                             seg_start, order);
+    count_launch(3);
     return cudaGetLastError();
 }
 

@@ -422,6 +422,115 @@ constexpr int R_WARPS = R_THREADS / 32;
 
 // One CTA per queued row: warp w evaluates centroids w, w + 8, ... in direct form with fp64
 // accumulation; the CTA then takes the smallest distance, lowest index on equality.
+// The same decision for RG queued rows per CTA at a time (rows of at most RG_MAX_D columns): the
+// rows sit in shared memory as fp64, so a centroid element is fetched and converted once for RG
+// rows and a row element is converted once for all K centroids -- the scan is bound by those
+// conversions and by the fp64 pipe, not by memory.  Warp w takes centroids w, w + 8, ... for all
+// rows of the group; lowest index on equality, as in the single-row form.
+constexpr int RG = 4;
+constexpr int RG_MAX_D = 1024;
+
+template <bool AFFINE>
+__device__ __forceinline__ void refine_body_grouped(const float *__restrict__ Y, int64_t N, int D, int K,
+                                                    const float *__restrict__ C, int32_t *labels,
+                                                    const int32_t *__restrict__ refine_rows, Control *ctl,
+                                                    const float *gamma, const float *beta, float *out,
+                                                    double *ys /* [RG][D] shared */)
+{
+    __shared__ double g_best[R_WARPS][RG];
+    __shared__ int g_idx[R_WARPS][RG];
+    __shared__ int g_label[RG];
+    __shared__ int64_t g_row[RG];
+    int count = ctl->refine_count;
+    if ((int64_t)count > N) count = (int)N;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctl->refined_total += count;
+        ctl->refined_last = count + ctl->cand_count;
+    }
+    const int lane = threadIdx.x & 31;
+    const int w = threadIdx.x >> 5;
+    for (int base = blockIdx.x * RG; base < count; base += gridDim.x * RG) {
+        const int nr = (count - base < RG) ? (count - base) : RG;
+        if (threadIdx.x < RG) {
+            int64_t row = (threadIdx.x < nr) ? (int64_t)refine_rows[base + threadIdx.x] : -1;
+            if (row >= N) row = -1;
+            g_row[threadIdx.x] = row;
+        }
+        __syncthreads();
+        for (int r = 0; r < RG; ++r) {
+            const int64_t row = g_row[r];
+            for (int j = threadIdx.x; j < D; j += R_THREADS)
+                ys[r * D + j] = (row >= 0) ? (double)Y[(size_t)row * D + j] : 0.0;
+        }
+        __syncthreads();
+        double best[RG];
+        int bk[RG];
+#pragma unroll
+        for (int r = 0; r < RG; ++r) {
+            best[r] = CUDART_INF;
+            bk[r] = K;
+        }
+        for (int k = w; k < K; k += R_WARPS) {
+            const float *c = C + (size_t)k * D;
+            double s[RG];
+#pragma unroll
+            for (int r = 0; r < RG; ++r) s[r] = 0.0;
+            for (int j = lane; j < D; j += 32) {
+                const double cv = (double)c[j];
+#pragma unroll
+                for (int r = 0; r < RG; ++r) {
+                    const double d = ys[r * D + j] - cv;
+                    s[r] = fma(d, d, s[r]);
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < RG; ++r) {
+                const double v = warp_sum(s[r]);
+                if (v < best[r]) {
+                    best[r] = v;
+                    bk[r] = k;
+                }
+            }
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int r = 0; r < RG; ++r) {
+                g_best[w][r] = best[r];
+                g_idx[w][r] = bk[r];
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < RG) {
+            const int r = threadIdx.x;
+            double b = g_best[0][r];
+            int k = g_idx[0][r];
+#pragma unroll
+            for (int q = 1; q < R_WARPS; ++q) {
+                if (g_best[q][r] < b || (g_best[q][r] == b && g_idx[q][r] < k)) {
+                    b = g_best[q][r];
+                    k = g_idx[q][r];
+                }
+            }
+            if (k >= K) k = 0;  // only when every distance is NaN
+            if (g_row[r] >= 0) labels[g_row[r]] = k;
+            g_label[r] = k;
+        }
+        __syncthreads();
+        if (AFFINE) {
+            for (int r = 0; r < RG; ++r) {
+                const int64_t row = g_row[r];
+                if (row < 0) continue;
+                const float *y = Y + (size_t)row * D;
+                const float *g = gamma + (size_t)g_label[r] * D;
+                const float *bb = beta + (size_t)g_label[r] * D;
+                float *o = out + (size_t)row * D;
+                for (int j = threadIdx.x; j < D; j += R_THREADS) o[j] = fmaf(g[j], y[j], bb[j]);
+            }
+        }
+        __syncthreads();
+    }
+}
+
 template <bool AFFINE>
 __device__ __forceinline__ void refine_body(const float *__restrict__ Y, int64_t N, int D, int K,
                                             const float *__restrict__ C, int32_t *labels,
@@ -509,8 +618,13 @@ __global__ void __launch_bounds__(R_THREADS) refine_kernel(const float *__restri
                                                            Control *ctl, const float *gamma,
                                                            const float *beta, float *out)
 {
-    refine_body<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out);
+    extern __shared__ double refine_rows_f64[];
+    if (D <= RG_MAX_D) refine_body_grouped<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out, refine_rows_f64);
+    else refine_body<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out);
 }
+
+// dynamic shared memory of the full-K exact pass: RG rows as fp64 where the grouped form applies
+static size_t refine_smem_bytes(int D) { return D <= RG_MAX_D ? (size_t)RG * D * sizeof(double) : 0; }
 
 cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *C,
                           int32_t *labels, const int32_t *refine_rows, Control *ctl,
@@ -518,10 +632,10 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
 {
     int blocks = (int)(N < 1184 ? N : 1184);
     if (out)
-        refine_kernel<true><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
+        refine_kernel<true><<<blocks, R_THREADS, refine_smem_bytes(D), s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
                                                          gamma, beta, out);
     else
-        refine_kernel<false><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
+        refine_kernel<false><<<blocks, R_THREADS, refine_smem_bytes(D), s>>>(Y, N, D, K, C, labels, refine_rows, ctl,
                                                           gamma, beta, out);
     count_launch();
     return cudaGetLastError();
@@ -664,7 +778,9 @@ __global__ void __launch_bounds__(R_THREADS) refine_both_kernel(
 {
     refine_candidates_body<AFFINE>(Y, N, D, K, C, labels, cand_rows, cand_list, ctl, gamma, beta, out, AFFINE);
     __syncthreads();   // (block 0's thread 0 updates the counters in both bodies, in this order)
-    refine_body<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out);
+    extern __shared__ double refine_rows_f64[];
+    if (D <= RG_MAX_D) refine_body_grouped<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out, refine_rows_f64);
+    else refine_body<AFFINE>(Y, N, D, K, C, labels, refine_rows, ctl, gamma, beta, out);
 }
 
 cudaError_t launch_refine_both(const float *Y, int64_t N, int D, int K, const float *C, int32_t *labels,
@@ -674,10 +790,10 @@ cudaError_t launch_refine_both(const float *Y, int64_t N, int D, int K, const fl
     int64_t want = (N + (RC_THREADS / 32) - 1) / (RC_THREADS / 32);
     int blocks = (int)(want < 1184 ? want : 1184);
     if (out)
-        refine_both_kernel<true><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
+        refine_both_kernel<true><<<blocks, R_THREADS, refine_smem_bytes(D), s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
                                                              refine_rows, ctl, gamma, beta, out);
     else
-        refine_both_kernel<false><<<blocks, R_THREADS, 0, s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
+        refine_both_kernel<false><<<blocks, R_THREADS, refine_smem_bytes(D), s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
                                                               refine_rows, ctl, gamma, beta, out);
     count_launch();
     return cudaGetLastError();

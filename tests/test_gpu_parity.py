@@ -244,6 +244,34 @@ def test_apply_column_split_falls_back_where_the_shape_does_not_allow_it():
     assert torch.equal(out, ref)
 
 
+@pytest.mark.parametrize("d,k", [(256, 32), (1024, 64), (64, 40)])
+def test_rows_between_two_centroids_are_decided_like_the_oracle(d, k):
+    """Rows placed next to the bisector of two centroids, with relative distance gaps from 1e-6 to
+    1e-4: all of them are undecidable for the tensor-core scores, and they straddle the margin
+    below which the exact pass leaves its fp32 pre-decision for fp64."""
+    rng = np.random.default_rng(d + k)
+    C = rng.normal(size=(k, d)).astype(np.float32)
+    n = 6000
+    a = rng.integers(0, k, size=n)
+    b = (a + 1 + rng.integers(0, k - 1, size=n)) % k
+    s = (10.0 ** rng.uniform(-6.9, -4.9, size=n)) * rng.choice([-1.0, 1.0], size=n)
+    Yq = ((C[a].astype(np.float64) + C[b]) / 2 + s[:, None] * (C[b].astype(np.float64) - C[a])).astype(np.float32)
+    G = rng.normal(size=(k, d)).astype(np.float32)
+    Bt = rng.normal(size=(k, d)).astype(np.float32)
+    want, lab, best, second = O.apply(Yq, C, G, Bt)
+    rel = (second - best) / second
+    assert (rel < 1e-3).mean() > 0.9 and (rel > 2e-6).mean() > 0.5   # the rows are where they were meant to be
+    ws = B.workspace("apply", n, d, k, "cuda")
+    out, glab = B.cat_apply(dev(Yq), dev(C), dev(G), dev(Bt), want_labels=True, ws=ws)
+    rep = B.cat_workspace_report(ws)
+    assert rep["refined_rows_last"] > n // 2      # they did go through the exact pass
+    _, n_diff = labels_match(host(glab), lab, best, second, "labels next to a bisector")
+    want2 = want if n_diff == 0 else O.affine_with_labels(Yq, host(glab), G, Bt)
+    close(host(out), want2, "outputs next to a bisector")
+    glab2 = B.cat_assign(dev(Yq), dev(C))
+    assert torch.equal(glab2, glab)
+
+
 def test_fit_fp16_and_tf32_operands_agree():
     """The default start lets cat_fit assign from an fp16 copy of the rows; an explicit start (here the
     same first K rows) keeps TF32 operands.  Labels are decided exactly either way."""

@@ -660,10 +660,20 @@ __device__ __forceinline__ void refine_candidates_body(
                                     reinterpret_cast<uintptr_t>(out)) & 15u) == 0);
     const int gw = blockIdx.x * (RC_THREADS / 32) + (threadIdx.x >> 5);
     const int nw = gridDim.x * (RC_THREADS / 32);
+    // A warp walks its rows one after the other, and each row is a chain of dependent loads (queue
+    // entry -> row and centroids -> label): the queue entry of the warp's next row is fetched while
+    // this row is worked on, and the row's fast label is requested together with its data.
+    int64_t next_row = (gw < count) ? (int64_t)cand_rows[gw] : -1;
+    uint64_t next_packed = (gw < count) ? cand_list[gw] : 0;
     for (int it = gw; it < count; it += nw) {
-        const int64_t row = cand_rows[it];
-        const uint64_t packed = cand_list[it];
+        const int64_t row = next_row;
+        const uint64_t packed = next_packed;
+        if (it + nw < count) {
+            next_row = cand_rows[it + nw];
+            next_packed = cand_list[it + nw];
+        }
         if (row < 0 || row >= N) continue;
+        const int fast = labels[row];
         int cand[4];
         const float *cp[4];
         int ncand = 0;   // the list is filled from the front: unused slots are at the end
@@ -744,8 +754,7 @@ __device__ __forceinline__ void refine_candidates_body(
         }
         if (bk >= K) bk = (cand[0] >= 0) ? cand[0] : 0;   // only when every distance is NaN
         // The fast pass has already written this row's output with the label it left in
-        // labels[row]; the row is rewritten only when the exact label differs.
-        const int fast = labels[row];
+        // labels[row] (read above); the row is rewritten only when the exact label differs.
         __syncwarp();
         if (lane == 0) labels[row] = bk;
         if (AFFINE && (bk != fast || !fast_output_valid)) {

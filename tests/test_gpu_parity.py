@@ -145,7 +145,7 @@ def _rand(seed, n, d):
 
 @pytest.mark.parametrize("n,d,k", [(1, 4, 1), (5, 1, 2), (127, 3, 3), (129, 7, 5), (300, 10, 9),
                                    (257, 1000, 17), (1000, 64, 65), (513, 36, 130), (64, 8, 64),
-                                   (2000, 20, 1), (900, 1024, 256), (700, 12, 512)])
+                                   (2000, 20, 1), (900, 1024, 256), (700, 12, 512), (600, 1540, 48), (300, 1100, 6)])
 def test_ragged_shapes_apply_and_fit(n, d, k):
     Yq = _rand(n * 7 + d, n, d)
     Yfp = (Yq * 1.1 + 0.1 * _rand(n + d + 1, n, d)).astype(np.float32)

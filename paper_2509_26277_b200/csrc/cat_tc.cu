@@ -29,7 +29,9 @@
 // For inference, streaming warps then read every row of the tile once more and write
 // gamma_l * y + beta_l for the fast label l; an undecided row is queued and the exact pass
 // rewrites its output.  The TMA producer may run at most one tile ahead of the streaming
-// warps, which bounds the bytes between a row's first read and its second.
+// warps, which bounds the bytes between a row's first read and its second.  A second form of the
+// same step (apply_split_kernel, selectable, off by default) shares one 128-row tile among the CTAs
+// of a cluster by columns and sums the partial scores through distributed shared memory.
 //
 // Every wait on an mbarrier or a progress counter is bounded (about 2 s): on a timeout the
 // CTA records CAT_ERR_DEVICE_TIMEOUT in the control block, all roles leave their loops,
@@ -1654,7 +1656,7 @@ cudaError_t launch_wait_selftest(Control *ctl, int limit_ms, cudaStream_t s)
 }
 
 // ---- column-split inference kernel: selection and launch
-static std::atomic<int> g_apply_split{0};   // 0 = chosen here, 1 = never, 2 / 4 = that cluster size where it applies
+static std::atomic<int> g_apply_split{0};   // 0 = chosen here (row tiles at present), 1 = never, 2 / 4 = that cluster size where it applies
 
 void set_apply_column_split(int cs) { g_apply_split.store((cs == 1 || cs == 2 || cs == 4) ? cs : 0, std::memory_order_relaxed); }
 int get_apply_column_split() { return g_apply_split.load(std::memory_order_relaxed); }

@@ -24,6 +24,36 @@ inline bool cuda_ok(cudaError_t e)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Programmatic dependent launch for the chains of short kernels (a Lloyd round is seven of them):
+// a kernel launched with launch_pdl may be scheduled while the previous kernel of its stream is
+// still running, which hides its launch latency.  Such a kernel calls pdl_enter() before anything
+// else: it lets its own dependents be scheduled early, then waits until the previous grid has
+// completed and its writes are visible -- so the kernels still run in stream order.  Both
+// instructions do nothing in a kernel that was launched the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_enter()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args &&...args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---------------------------------------------------------------- workspace layouts
 // Control block at the start of every workspace (device memory).
 struct Control {

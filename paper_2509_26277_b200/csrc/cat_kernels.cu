@@ -785,6 +785,7 @@ __global__ void __launch_bounds__(R_THREADS) refine_both_kernel(
     const int32_t *__restrict__ cand_rows, const uint64_t *__restrict__ cand_list,
     const int32_t *__restrict__ refine_rows, Control *ctl, const float *gamma, const float *beta, float *out)
 {
+    pdl_enter();
     refine_candidates_body<AFFINE>(Y, N, D, K, C, labels, cand_rows, cand_list, ctl, gamma, beta, out, AFFINE);
     __syncthreads();   // (block 0's thread 0 updates the counters in both bodies, in this order)
     extern __shared__ double refine_rows_f64[];
@@ -799,11 +800,11 @@ cudaError_t launch_refine_both(const float *Y, int64_t N, int D, int K, const fl
     int64_t want = (N + (RC_THREADS / 32) - 1) / (RC_THREADS / 32);
     int blocks = (int)(want < 1184 ? want : 1184);
     if (out)
-        refine_both_kernel<true><<<blocks, R_THREADS, refine_smem_bytes(D), s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
-                                                             refine_rows, ctl, gamma, beta, out);
+        launch_pdl(refine_both_kernel<true>, dim3(blocks), dim3(R_THREADS), refine_smem_bytes(D), s, Y, N, D, K, C, labels,
+                   cand_rows, cand_list, refine_rows, ctl, gamma, beta, out);
     else
-        refine_both_kernel<false><<<blocks, R_THREADS, refine_smem_bytes(D), s>>>(Y, N, D, K, C, labels, cand_rows, cand_list,
-                                                              refine_rows, ctl, gamma, beta, out);
+        launch_pdl(refine_both_kernel<false>, dim3(blocks), dim3(R_THREADS), refine_smem_bytes(D), s, Y, N, D, K, C, labels,
+                   cand_rows, cand_list, refine_rows, ctl, gamma, beta, out);
     count_launch();
     return cudaGetLastError();
 }

@@ -56,6 +56,7 @@ __global__ void __launch_bounds__(SORT_BLOCK) label_hist_kernel(const int32_t *_
                                                                  const int32_t *__restrict__ prev, int64_t N, int K,
                                                                  int KK, uint32_t *__restrict__ blk_hist)
 {
+    pdl_enter();
     extern __shared__ uint32_t hist[];   // [KK]
     for (int k = threadIdx.x; k < KK; k += SORT_BLOCK) hist[k] = 0;
     __syncthreads();
@@ -71,6 +72,7 @@ __global__ void __launch_bounds__(SORT_BLOCK) label_hist_kernel(const int32_t *_
 __global__ void __launch_bounds__(256) label_scan_blocks_kernel(uint32_t *__restrict__ blk_hist, int nblk, int KK,
                                                                  uint32_t *__restrict__ key_total)
 {
+    pdl_enter();
     const int k = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
     const int lane = threadIdx.x & 31;
     if (k >= KK) return;
@@ -176,6 +178,7 @@ __global__ void __launch_bounds__(SORT_BLOCK) label_scatter_kernel(const int32_t
                                                                     int32_t *__restrict__ seg_start,
                                                                     int32_t *__restrict__ order)
 {
+    pdl_enter();
     extern __shared__ uint32_t scatter_smem[];   // [KK] key offsets, then [32][KK] 16-bit warp histograms
     __shared__ uint32_t wsum[33];
     uint32_t *key_off = scatter_smem;
@@ -267,6 +270,7 @@ __device__ __forceinline__ void seg_accumulate(double (&a0)[4], double (&a1)[4],
 template <int MODE, int VEC>
 __global__ void __launch_bounds__(SEG_THREADS) segment_sums_kernel(SegParams p)
 {
+    pdl_enter();
     __shared__ int32_t rows_s[128];
     __shared__ double red_s[SEG_THREADS * VEC];
     const int nseg_total = p.seg_start[p.K];
@@ -427,6 +431,7 @@ __global__ void __launch_bounds__(1024) centroid_update_kernel(const double *__r
                                                               float *__restrict__ cnorm, const float *__restrict__ scale,
                                                               __half *__restrict__ Ch, Control *ctl)
 {
+    pdl_enter();
     __shared__ double red[32];
     const int k = blockIdx.x;
     if (k == 0 && threadIdx.x == 0) {
@@ -491,8 +496,8 @@ cudaError_t launch_label_sort(const int32_t *labels, const int32_t *prev, int64_
                               int32_t *seg_start, int32_t *order, cudaStream_t s)
 {
     const int KK = prev ? 2 * K : K;
-    label_hist_kernel<<<g.nblk, SORT_BLOCK, (size_t)KK * sizeof(uint32_t), s>>>(labels, prev, N, K, KK, blk_hist);
-    label_scan_blocks_kernel<<<(KK * 32 + 255) / 256, 256, 0, s>>>(blk_hist, g.nblk, KK, key_total);
+    launch_pdl(label_hist_kernel, dim3(g.nblk), dim3(SORT_BLOCK), (size_t)KK * sizeof(uint32_t), s, labels, prev, N, K, KK, blk_hist);
+    launch_pdl(label_scan_blocks_kernel, dim3((KK * 32 + 255) / 256), dim3(256), 0, s, blk_hist, g.nblk, KK, key_total);
     // (the scan over the keys -- key offsets, segment table, cluster sizes -- runs inside the scatter
     // kernel: every CTA needs the offsets, CTA 0 publishes the tables)
     const size_t sc_smem = (size_t)KK * sizeof(uint32_t) + (size_t)32 * KK * sizeof(uint16_t);
@@ -501,9 +506,8 @@ cudaError_t launch_label_sort(const int32_t *labels, const int32_t *prev, int64_
                                              (int)sc_smem);
         if (e != cudaSuccess) return e;
     }
-    label_scatter_kernel<<<g.nblk, SORT_BLOCK, sc_smem, s>>>(labels, prev, N, K, KK, blk_hist, key_total, g.seg_rows,
-                                                             prev ? 2 * N : N, prev ? 1 : 0, counts, cluster_start,
-                                                             seg_start, order);
+    launch_pdl(label_scatter_kernel, dim3(g.nblk), dim3(SORT_BLOCK), sc_smem, s, labels, prev, N, K, KK, blk_hist, key_total,
+               g.seg_rows, prev ? 2 * N : N, prev ? 1 : 0, counts, cluster_start, seg_start, order);
     count_launch(3);
     return cudaGetLastError();
 }
@@ -518,9 +522,9 @@ static cudaError_t launch_segment_sums_mode(const SegParams &p, const SegGeom &g
     const unsigned gx = (unsigned)(g.max_segs < 1184 ? g.max_segs : 1184);
     dim3 grid(gx, (unsigned)((units + SEG_THREADS - 1) / SEG_THREADS));
     if (vec)
-        segment_sums_kernel<MODE, 4><<<grid, SEG_THREADS, 0, s>>>(p);
+        launch_pdl(segment_sums_kernel<MODE, 4>, grid, dim3(SEG_THREADS), 0, s, p);
     else
-        segment_sums_kernel<MODE, 1><<<grid, SEG_THREADS, 0, s>>>(p);
+        launch_pdl(segment_sums_kernel<MODE, 1>, grid, dim3(SEG_THREADS), 0, s, p);
     count_launch();
     return cudaGetLastError();
 }
@@ -580,8 +584,8 @@ cudaError_t launch_centroid_update(const double *part, const int32_t *seg_start,
 {
     // one thread per column where the row is short enough: the loads of a column depend on each other
     const int threads = D >= 1024 ? 1024 : (D >= 512 ? 512 : 256);
-    centroid_update_kernel<<<K, threads, 0, s>>>(part, seg_start, counts, D, K, sums, C, cnorm, scale,
-                                             reinterpret_cast<__half *>(Ch), ctl);
+    launch_pdl(centroid_update_kernel, dim3(K), dim3(threads), 0, s, part, seg_start, counts, D, K, sums, C, cnorm, scale,
+               reinterpret_cast<__half *>(Ch), ctl);
     count_launch();
     return cudaGetLastError();
 }

@@ -627,6 +627,7 @@ template <bool AFFINE, bool PAIR, bool HALF, bool SHORT>
 __global__ void __launch_bounds__(AFFINE ? TC_THREADS_AFFINE : TC_THREADS_LABELS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcParams p)
 {
+    pdl_enter();
     extern __shared__ unsigned char smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle
     const uint32_t raw = smem_u32(smem_raw);
@@ -1832,13 +1833,15 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
     cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = pair ? 2 : 1;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // (the kernel starts with pdl_enter)
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
 
     cudaError_t e;
 #define CAT_TC_LAUNCH(AFF, PR, HF, SH)                                                                                      \

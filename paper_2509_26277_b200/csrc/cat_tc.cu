@@ -337,24 +337,6 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, uint32_t fmt)
     return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// Optional timeline of the first two CTAs (compiled in only with -DCAT_TC_TRACE): globaltimer
-// stamps per role and tile, read back with cat_tc_trace_read.
-#ifdef CAT_TC_TRACE
-constexpr int TC_TRACE_TILES = 16;
-constexpr int TC_TRACE_EVENTS = 8;
-__device__ unsigned long long g_tc_trace[2][TC_TRACE_TILES][TC_TRACE_EVENTS];
-#ifndef CAT_TC_TRACE_FIRST
-#define CAT_TC_TRACE_FIRST 0
-#endif
-#define TC_TRACE(ti, ev)                                                                               \
-    do {                                                                                               \
-        if (blockIdx.x < 2 && (ti) >= CAT_TC_TRACE_FIRST && (ti) < CAT_TC_TRACE_FIRST + TC_TRACE_TILES) \
-            g_tc_trace[blockIdx.x][(ti) - CAT_TC_TRACE_FIRST][ev] = global_timer();                    \
-    } while (0)
-#else
-#define TC_TRACE(ti, ev) do { } while (0)
-#endif
-
 struct TcParams {
     const float *Y;
     const float *cnorm;
@@ -467,60 +449,9 @@ __device__ __forceinline__ bool tc_decide(const TcParams &p, int64_t row, float4
 
 // One warp streams one row (1024 columns per step, all loads of a step in flight together):
 // out = gamma_l * y + beta_l for the fast label l, written whether or not the label is
-// certain (an undecided row is queued and the exact pass rewrites it); the row norm needed
-// by the certainty test is accumulated on the way.
-__device__ __forceinline__ void stream_row(const TcParams &p, int64_t row, float4 keys, float cmax2, int lane)
-{
-    const int D4 = p.D >> 2;
-    const int l = key_label(keys.x, p.K);
-    const float4 *y4 = reinterpret_cast<const float4 *>(p.Y) + (size_t)row * D4 + lane;
-    const float4 *g4 = reinterpret_cast<const float4 *>(p.gamma) + (size_t)l * D4 + lane;
-    const float4 *b4 = reinterpret_cast<const float4 *>(p.beta) + (size_t)l * D4 + lane;
-    float4 *o4 = reinterpret_cast<float4 *>(p.out) + (size_t)row * D4 + lane;
-    float ysq = 0.f;
-#pragma unroll 1
-    for (int h = 0; h < D4; h += 256) {
-        float4 y[8], g[8], bb[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int c = h + 32 * q;
-            if (c + lane < D4) {
-                y[q] = __ldcs(y4 + c);
-                g[q] = __ldg(g4 + c);
-                bb[q] = __ldg(b4 + c);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int c = h + 32 * q;
-            if (c + lane < D4) {
-                float4 v;
-                v.x = fmaf(g[q].x, y[q].x, bb[q].x);
-                v.y = fmaf(g[q].y, y[q].y, bb[q].y);
-                v.z = fmaf(g[q].z, y[q].z, bb[q].z);
-                v.w = fmaf(g[q].w, y[q].w, bb[q].w);
-                __stcs(o4 + c, v);
-                ysq = fmaf(y[q].x, y[q].x, ysq);
-                ysq = fmaf(y[q].y, y[q].y, ysq);
-                ysq = fmaf(y[q].z, y[q].z, ysq);
-                ysq = fmaf(y[q].w, y[q].w, ysq);
-            }
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
-    if (lane == 0) {
-        // the row norm enters the bound slightly over-estimated
-        const float e = tc_error_bound(p.D, ysq * 1.0001f, cmax2);
-        p.labels[row] = l;
-        tc_decide(p, row, keys, e);
-    }
-}
-
-// Streaming of one row without the certainty test: out = gamma_l * y + beta_l, returns ||y||^2
-// (complete in every lane).  The column-split kernel decides certainty in its score warps, which
-// leaves the streaming loop the registers for 24 loads per lane in flight and little else.
-__device__ __forceinline__ float stream_row_lean(const TcParams &p, int64_t row, int l, int lane)
+// certain (an undecided row is queued and the exact pass rewrites it).  Returns ||y||^2,
+// accumulated on the way and complete in every lane.
+__device__ __forceinline__ float stream_row_affine(const TcParams &p, int64_t row, int l, int lane)
 {
     const int D4 = p.D >> 2;
     const float4 *y4 = reinterpret_cast<const float4 *>(p.Y) + (size_t)row * D4 + lane;
@@ -562,7 +493,22 @@ __device__ __forceinline__ float stream_row_lean(const TcParams &p, int64_t row,
     return ysq;
 }
 
-// The same for short rows (D < 128): a row takes only G = 1 .. 16 lanes, so a warp streams all
+// The row-tile kernel decides certainty right after streaming the row, in the streaming warp.
+// (The column-split kernel decides in its score warps instead: its streaming loop has no
+// register to spare.)
+__device__ __forceinline__ void stream_row(const TcParams &p, int64_t row, float4 keys, float cmax2, int lane)
+{
+    const int l = key_label(keys.x, p.K);
+    const float ysq = stream_row_affine(p, row, l, lane);
+    if (lane == 0) {
+        // the row norm enters the bound slightly over-estimated
+        const float e = tc_error_bound(p.D, ysq * 1.0001f, cmax2);
+        p.labels[row] = l;
+        tc_decide(p, row, keys, e);
+    }
+}
+
+// The same for short rows (D < 128): a row takes only G = 1 .. 32 lanes, so a warp streams all
 // of its rows of the tile (ew, ew + TC_STREAM_WARPS, ...) in one step, 32 / G rows per load slot.
 __device__ __forceinline__ void stream_rows_short(const TcParams &p, int64_t row0, const float4 *tile_keys, int ew,
                                                   float cmax2, int lane)
@@ -605,7 +551,7 @@ __device__ __forceinline__ void stream_rows_short(const TcParams &p, int64_t row
                 ysq = fmaf(y[q].x, y[q].x, fmaf(y[q].y, y[q].y, fmaf(y[q].z, y[q].z, y[q].w * y[q].w)));
             }
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1)
+            for (int o = 16; o > 0; o >>= 1)
                 if (o < G) ysq += __shfl_xor_sync(0xffffffffu, ysq, o);
             if ((act & (1u << q)) && c == 0) {
                 const float4 keys = tile_keys[r];
@@ -719,8 +665,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     }
                     for (int sl = 0; sl < nslabs; ++sl) {
                         if (!mbar_wait(smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
-                        if (sl == 0) TC_TRACE(ti, 0);
-                        if (sl == nslabs - 1) TC_TRACE(ti, 1);
                         const uint32_t a_dst = tiles_base + (uint32_t)(s * TC_A_BYTES);
                         if (PAIR) {
                             // both CTAs report to the barrier of the MMA-issuing CTA
@@ -788,8 +732,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                         // issuing thread's own instruction count is what paces the MMAs)
                         if (!mbar_wait(smem_u32(&sh.b_full[sb]), phb, abort_flag, p.ctl)) { ok = false; break; }
                         if (!mbar_wait(smem_u32(&sh.a_full[sa]), pha, abort_flag, p.ctl)) { ok = false; break; }
-                        if (sl == 0) TC_TRACE(ti, 2);
-                        if (sl == nslabs - 1) TC_TRACE(ti, 3);
                         tc_fence_after();
                         // (the start address sits in the low bits of the descriptor, in 16-byte units)
                         const uint64_t adesc = AFFINE ? make_smem_desc(tiles_base + (uint32_t)(sa * TC_A_BYTES))
@@ -856,7 +798,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             if (!AFFINE && row0 + quarter * 32 + lane < p.N) yn2 = p.ynorm2[row0 + quarter * 32 + lane];
             if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
             tc_fence_after();
-            if (quarter == 0 && lane == 0) TC_TRACE(ti, 4);
             const float coef = coef_c * rinv;
             float b1 = TC_KEY_INIT, b2 = TC_KEY_INIT, b3 = TC_KEY_INIT, b4 = TC_KEY_INIT;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
@@ -875,7 +816,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 for (int j = 0; j < 16; ++j)
                     key_insert(make_key(fmaf(coef, __uint_as_float(rb[j]), sh.cn[c + 16 + j]), c + 16 + j), b1, b2, b3, b4);
             }
-            if (quarter == 0 && lane == 0) TC_TRACE(ti, 5);
             // accumulator buffer b may be overwritten from here on
             tc_fence_before();
             __syncwarp();
@@ -911,7 +851,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             const uint32_t ph = (ti >> 1) & 1u;
             const int64_t row0 = PAIR ? (unit * 2 + rank) * TC_BM : unit * TC_BM;
             if (!mbar_wait_warp(smem_u32(&sh.lab_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
-            if (ew == 0 && lane == 0) TC_TRACE(ti, 6);
             if (SHORT) {
                 stream_rows_short(p, row0, sh.top_key[b], ew, cmax2, lane);
                 __syncwarp();
@@ -925,7 +864,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                 }
             }
             __syncwarp();
-            if (ew == 0 && lane == 0) TC_TRACE(ti, 7);
             if (lane == 0) mbar_arrive(smem_u32(&sh.lab_empty[b]));
         }
     }
@@ -1124,8 +1062,6 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     }
                     for (int sl = 0; sl < nslabs; ++sl) {
                         if (!mbar_wait(smem_u32(&sh.a_empty[s]), ph ^ 1u, abort_flag, p.ctl)) { ok = false; break; }
-                        if (sl == 0) TC_TRACE(ti, 0);
-                        if (sl == nslabs - 1) TC_TRACE(ti, 1);
                         const uint32_t full = smem_u32(&sh.a_full[s]);
                         mbar_arrive_expect_tx(full, (uint32_t)TC_A_BYTES);
                         tma_load_2d(tiles_base + (uint32_t)(s * TC_A_BYTES), &mapA, full, (slab0 + sl) * 32, row0);
@@ -1174,8 +1110,6 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     for (int sl = 0; sl < nslabs; ++sl) {
                         if (!mbar_wait(smem_u32(&sh.b_full[sb]), phb, abort_flag, p.ctl)) { ok = false; break; }
                         if (!mbar_wait(smem_u32(&sh.a_full[sa]), pha, abort_flag, p.ctl)) { ok = false; break; }
-                        if (sl == 0) TC_TRACE(ti, 2);
-                        if (sl == nslabs - 1) TC_TRACE(ti, 3);
                         tc_fence_after();
                         const uint64_t adesc = make_smem_desc(tiles_base + (uint32_t)(sa * TC_A_BYTES));
                         const uint64_t bdesc = make_smem_desc(b_base + (uint32_t)(sb * b_bytes));
@@ -1208,7 +1142,6 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             const uint32_t ph = (ti >> 1) & 1u;
             if (!mbar_wait_warp(smem_u32(&sh.tmem_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
             tc_fence_after();
-            if (quarter == 0 && lane == 0) TC_TRACE(ti, 4);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.npad);
             uint32_t ra[16], rb[16];
             // ---- send: the peers' centroid ranges of this CTA's partial scores
@@ -1267,7 +1200,6 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                         key_insert(make_key(fmaf(-2.f, acc[j] + __uint_as_float(ra[j]), sh.cn[k0 + c + j]), k0 + c + j), b1, b2, b3, b4);
                 }
             }
-            if (quarter == 0 && lane == 0) TC_TRACE(ti, 5);
             // accumulator buffer b and the exchange buffer are free from here on
             tc_fence_before();
             // (no separate fence: __syncwarp orders the lanes, the arrival below releases at cluster scope)
@@ -1336,18 +1268,16 @@ apply_split_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             const uint32_t ph = (ti >> 1) & 1u;
             const int64_t row0 = unit * TC_BM + (int64_t)crank * RP;
             if (!mbar_wait_warp(smem_u32(&sh.lab_full[b]), ph, abort_flag, p.ctl)) { ok = false; break; }
-            if (ew == 0 && lane == 0) TC_TRACE(ti, 6);
             for (int rl = ew; rl < RP; rl += TCS_STREAM_WARPS) {
                 const int64_t row = row0 + rl;
                 if (row < p.N) {
-                    const float ysq = stream_row_lean(p, row, key_label(sh.top_key[b][rl].x, p.K), lane);
+                    const float ysq = stream_row_affine(p, row, key_label(sh.top_key[b][rl].x, p.K), lane);
                     if (lane == 0) sh.row_norm[b][rl] = ysq;
                 }
                 __syncwarp();
                 if (lane == 0) atomicAdd(&sh.rows_streamed, 1);
             }
             __syncwarp();
-            if (ew == 0 && lane == 0) TC_TRACE(ti, 7);
             if (lane == 0) mbar_arrive(smem_u32(&sh.lab_empty[b]));
         }
     }
@@ -1438,15 +1368,19 @@ __global__ void __launch_bounds__(256) half_shadow_kernel(const float *__restric
     const int rows_per_cta = 256 / G;
     const int sub = threadIdx.x / G, c0 = threadIdx.x % G;
     float cta_max = 0.f;
-    for (int64_t row = (int64_t)blockIdx.x * rows_per_cta + sub; row < N; row += (int64_t)gridDim.x * rows_per_cta) {
-        const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)row * D);
+    // The trip count is the same for every thread of the CTA (the shuffles below name all 32
+    // lanes); a thread whose row lies beyond N goes through the loop with loads and stores off.
+    for (int64_t base = (int64_t)blockIdx.x * rows_per_cta; base < N; base += (int64_t)gridDim.x * rows_per_cta) {
+        const int64_t row = base + sub;
+        const bool live = row < N;
+        const float4 *y4 = reinterpret_cast<const float4 *>(Y + (size_t)(live ? row : 0) * D);
         float s = 0.f, m = 0.f;
         for (int c = c0; c < D4; c += 8 * G) {
             float4 v[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int cc = c + u * G;
-                v[u] = (cc < D4) ? __ldg(y4 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+                v[u] = (live && cc < D4) ? __ldg(y4 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -1470,6 +1404,7 @@ __global__ void __launch_bounds__(256) half_shadow_kernel(const float *__restric
         if (sh > 100) sh = 100;
         if (sh < -100) sh = -100;
         const float sc = ldexpf(1.f, sh);
+        if (!live) continue;
         if (c0 == 0) {
             ynorm2[row] = s * 1.0001f;
             rinv[row] = ldexpf(1.f, -sh);
@@ -1870,10 +1805,3 @@ cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const floa
 }
 
 }  // namespace cat
-
-#ifdef CAT_TC_TRACE
-extern "C" int cat_tc_trace_read(unsigned long long *host_out)
-{
-    return (int)cudaMemcpyFromSymbol(host_out, cat::g_tc_trace, sizeof(cat::g_tc_trace));
-}
-#endif

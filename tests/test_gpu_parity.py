@@ -145,7 +145,9 @@ def _rand(seed, n, d):
 
 @pytest.mark.parametrize("n,d,k", [(1, 4, 1), (5, 1, 2), (127, 3, 3), (129, 7, 5), (300, 10, 9),
                                    (257, 1000, 17), (1000, 64, 65), (513, 36, 130), (64, 8, 64),
-                                   (2000, 20, 1), (900, 1024, 256), (700, 12, 512), (600, 1540, 48), (300, 1100, 6)])
+                                   (2000, 20, 1), (900, 1024, 256), (700, 12, 512), (600, 1540, 48), (300, 1100, 6),
+                                   # N not a multiple of the rows a warp shares when a row takes fewer than 32 lanes
+                                   (1001, 64, 65), (67, 8, 64), (515, 32, 40), (333, 120, 33)])
 def test_ragged_shapes_apply_and_fit(n, d, k):
     Yq = _rand(n * 7 + d, n, d)
     Yfp = (Yq * 1.1 + 0.1 * _rand(n + d + 1, n, d)).astype(np.float32)
@@ -244,7 +246,7 @@ def test_apply_column_split_falls_back_where_the_shape_does_not_allow_it():
     assert torch.equal(out, ref)
 
 
-@pytest.mark.parametrize("d,k", [(256, 32), (1024, 64), (64, 40)])
+@pytest.mark.parametrize("d,k", [(256, 32), (1024, 64), (64, 40), (120, 33), (68, 40)])
 def test_rows_between_two_centroids_are_decided_like_the_oracle(d, k):
     """Rows placed next to the bisector of two centroids, with relative distance gaps from 1e-6 to
     1e-4: all of them are undecidable for the tensor-core scores, and they straddle the margin

@@ -52,12 +52,25 @@ enum {
 #define CAT_MAX_K 512
 #define CAT_MAX_D 16384
 
-/* Diagnostics of one cat_fit call, written to device memory (all int64). */
+/* Diagnostics of one cat_fit_from call, written to device memory.  The first four words are
+ * always filled.  The per-assignment records cost an extra pass over Yq after every assignment
+ * (the `iters` assignments of the Lloyd rounds and the final one, Algorithm 1 with K-Means as
+ * the cluster model), so a fit that asks for them is slower than one that passes diag = NULL.
+ * Assignment t is recorded at index t for t < CAT_DIAG_MAX_ROUNDS - 1; the final assignment is
+ * always recorded, at index min(iters, CAT_DIAG_MAX_ROUNDS - 1). */
+#define CAT_DIAG_MAX_ROUNDS 64
 typedef struct cat_fit_diag {
     int64_t refined_rows_total;   /* rows whose label needed the exact fp64 pass, summed over all assignments */
     int64_t refined_rows_final;   /* same, final assignment only */
     int64_t empty_clusters_final; /* clusters with no rows in the final assignment */
     int64_t device_status;        /* CAT_OK or CAT_ERR_DEVICE_TIMEOUT */
+    int64_t assignments_recorded; /* min(iters + 1, CAT_DIAG_MAX_ROUNDS) */
+    int64_t undecided_rows[CAT_DIAG_MAX_ROUNDS]; /* rows the fast scores could not decide (sent to the exact pass) */
+    int64_t near_tie_rows[CAT_DIAG_MAX_ROUNDS];  /* rows whose two nearest centroids are within 1e-6 relative of each
+                                                    other in squared distance (fp64 direct form) */
+    double objective[CAT_DIAG_MAX_ROUNDS];       /* sum_i ||Yq_i - c_label(i)||^2 against the centroids the assignment
+                                                    used, fp64; the order of the additions is not fixed, so the last
+                                                    bits vary from run to run */
 } cat_fit_diag_t;
 
 /* ---- the two calls of the hot path ------------------------------------ */
@@ -132,6 +145,37 @@ cat_status_t cat_apply_blend(const float *Yq, int64_t N, int32_t D, int32_t K,
 cat_status_t cat_assign(const float *Yq, int64_t N, int32_t D, int32_t K,
                         const float *centroids, int32_t *labels_out,
                         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * cat_assign that also hands out what its fast pass saw, so that the label decision can be
+ * audited from outside (Alg. 2 step 2; the decision rule is the library's own: a row's label is
+ * taken from fast scores t_k = ||c_k||^2 - 2 y.c_k when the two smallest are more than 2e apart,
+ * e being a bound on the error of a fast score, and from fp64 direct-form distances otherwise).
+ * Every array of `scores` has N entries and may be NULL:
+ *   best, second  the two smallest fast scores of the row.  On the tensor-core path a score
+ *                 carries the index of its centroid in the low 8 bits of its fp32 pattern.
+ *   bound         e for this row: |fast score - exact score| <= e for every centroid (the
+ *                 tensor-core bound includes the index packing).
+ *   label         the centroid of `best`, i.e. the label before the exact pass.
+ * labels_out receives the final labels as cat_assign gives them.
+ * flags: CAT_ASSIGN_FP16_OPERANDS runs the tensor-core contraction on an fp16 copy of the rows
+ * (per-row power-of-two scale) and of the centroids, as cat_fit does for its Lloyd rounds; it
+ * needs D % 8 == 0 and K <= 256 (CAT_ERR_UNSUPPORTED otherwise) and a workspace of
+ * cat_fit_workspace_bytes(N, D, K); the centroids must not exceed the largest magnitude of Yq.
+ * Without flags the workspace is cat_apply_workspace_bytes(N, D, K).
+ */
+typedef struct cat_fast_scores {
+    float *best;
+    float *second;
+    float *bound;
+    int32_t *label;
+} cat_fast_scores_t;
+#define CAT_ASSIGN_FP16_OPERANDS 1
+
+cat_status_t cat_assign_scores(const float *Yq, int64_t N, int32_t D, int32_t K,
+                               const float *centroids, int32_t *labels_out,
+                               const cat_fast_scores_t *scores, int32_t flags,
+                               void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * cat_assign without any workspace: the same labels as cat_assign, for callers that

@@ -23,10 +23,18 @@ STATUS_NAMES = {0: "CAT_OK", 1: "CAT_ERR_NULL", 2: "CAT_ERR_SHAPE", 3: "CAT_ERR_
                 7: "CAT_ERR_UNSUPPORTED"}
 MAX_K = 512
 MAX_D = 16384
+DIAG_MAX_ROUNDS = 64                       # CAT_DIAG_MAX_ROUNDS
+_DIAG_WORDS = 5 + 3 * DIAG_MAX_ROUNDS      # cat_fit_diag_t in 8-byte words
+ASSIGN_FP16_OPERANDS = 1                   # CAT_ASSIGN_FP16_OPERANDS
+
+
+class _FastScores(ctypes.Structure):       # cat_fast_scores_t
+    _fields_ = [("best", ctypes.c_void_p), ("second", ctypes.c_void_p), ("bound", ctypes.c_void_p),
+                ("label", ctypes.c_void_p)]
 
 EXPORTS = [
     "cat_fit_workspace_bytes", "cat_fit", "cat_fit_from", "cat_apply_workspace_bytes",
-    "cat_apply", "cat_apply_blend", "cat_assign", "cat_assign_noalloc", "cat_cluster_sums",
+    "cat_apply", "cat_apply_blend", "cat_assign", "cat_assign_scores", "cat_assign_noalloc", "cat_cluster_sums",
     "cat_centroids_from_sums",
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
@@ -81,6 +89,8 @@ def lib():
     L.cat_apply.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     L.cat_apply_blend.argtypes = [vp, i64, i32, i32, vp, vp, vp, f32, vp, vp, vp, sz, vp]
     L.cat_assign.argtypes = [vp, i64, i32, i32, vp, vp, vp, sz, vp]
+    L.cat_assign_scores.argtypes = [vp, i64, i32, i32, vp, vp, ctypes.POINTER(_FastScores), i32, vp, sz, vp]
+    L.cat_assign_scores.restype = ctypes.c_int
     L.cat_assign_noalloc.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     L.cat_assign_noalloc.restype = ctypes.c_int
     L.cat_cluster_sums.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, sz, vp]
@@ -182,7 +192,7 @@ def cat_fit(Yq, Yfp, K: int, iters: int, init_centroids=None, want_labels=True, 
     G = torch.empty((K, D), dtype=torch.float32, device=dev)
     B = torch.empty((K, D), dtype=torch.float32, device=dev)
     labels = torch.empty((N,), dtype=torch.int32, device=dev) if want_labels else None
-    diag = torch.zeros((4,), dtype=torch.int64, device=dev) if want_diag else None
+    diag = torch.zeros((_DIAG_WORDS,), dtype=torch.int64, device=dev) if want_diag else None
     ws = workspace("fit", N, D, K, dev) if ws is None else ws
     st = lib().cat_fit_from(_dev(Yq, torch.float32, None, "Yq"), _dev(Yfp, torch.float32, (N, D), "Yfp"),
                             N, D, K, iters, _dev(init_centroids, torch.float32, (K, D), "init_centroids"),
@@ -191,9 +201,14 @@ def cat_fit(Yq, Yfp, K: int, iters: int, init_centroids=None, want_labels=True, 
                             ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream())
     _check(st, "cat_fit")
     if want_diag:
-        d = diag.tolist()
-        return C, G, B, labels, dict(refined_rows_total=d[0], refined_rows_final=d[1],
-                                     empty_clusters_final=d[2], device_status=d[3])
+        d = diag.cpu()
+        n, R = int(d[4]), DIAG_MAX_ROUNDS
+        return C, G, B, labels, dict(refined_rows_total=int(d[0]), refined_rows_final=int(d[1]),
+                                     empty_clusters_final=int(d[2]), device_status=int(d[3]),
+                                     assignments_recorded=n,
+                                     undecided_rows=d[5:5 + n].tolist(),
+                                     near_tie_rows=d[5 + R:5 + R + n].tolist(),
+                                     objective=d[5 + 2 * R:5 + 2 * R + n].view(torch.float64).tolist())
     return C, G, B, labels
 
 
@@ -255,6 +270,29 @@ def cat_assign(Yq, centroids, ws=None):
                           ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream())
     _check(st, "cat_assign")
     return labels
+
+
+def cat_assign_scores(Yq, centroids, fp16_operands: bool = False, ws=None):
+    """cat_assign_scores: returns (labels, dict(best, second, bound, label)) -- the final labels and what
+    the fast pass saw for every row (see cat.h)."""
+    N, D = Yq.shape
+    K = centroids.shape[0]
+    dev = Yq.device
+    labels = torch.empty((N,), dtype=torch.int32, device=dev)
+    rec = dict(best=torch.empty((N,), dtype=torch.float32, device=dev),
+               second=torch.empty((N,), dtype=torch.float32, device=dev),
+               bound=torch.empty((N,), dtype=torch.float32, device=dev),
+               label=torch.empty((N,), dtype=torch.int32, device=dev))
+    fs = _FastScores(rec["best"].data_ptr(), rec["second"].data_ptr(), rec["bound"].data_ptr(),
+                     rec["label"].data_ptr())
+    if ws is None:
+        ws = workspace("fit" if fp16_operands else "apply", N, D, K, dev)
+    st = lib().cat_assign_scores(_dev(Yq, torch.float32, None, "Yq"), N, D, K,
+                                 _dev(centroids, torch.float32, (K, D), "centroids"), _dev(labels, torch.int32),
+                                 ctypes.byref(fs), ASSIGN_FP16_OPERANDS if fp16_operands else 0,
+                                 ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream())
+    _check(st, "cat_assign_scores")
+    return labels, rec
 
 
 NOALLOC_MAX_ROWS = 262144

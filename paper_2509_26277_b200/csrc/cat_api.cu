@@ -38,6 +38,8 @@ static void carve_assign_into(Carver &c, AssignWs &w, int64_t N, int D, int K)
     w.ynorm2 = c.take<float>((size_t)N);
     w.cand_rows = c.take<int32_t>((size_t)N);
     w.cand_list = c.take<uint64_t>((size_t)N);
+    w.ch = c.take<uint16_t>((size_t)K * D);
+    w.hscale = c.take<float>(4);
 }
 
 AssignWs carve_assign(void *base, int64_t N, int D, int K)
@@ -110,20 +112,30 @@ static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const fl
                                const float *beta, float *out, cudaStream_t s,
                                bool row_norms_ready = false, bool top_level = true,
                                const void *Yh = nullptr, void *Ch = nullptr, const float *hscale = nullptr,
-                               bool centroids_ready = false)
+                               bool centroids_ready = false, const FastOut *fast = nullptr)
 {
     // centroids_ready: the centroid update that produced C has already left its norms, its fp16
     // copy and empty exact-pass queues in the workspace
     if (!centroids_ready) CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s, top_level));
-    if (use_tensor_path(N, D, K)) {
+    if (out && use_tensor_path(N, D, K) && choose_apply_form(N, D, K) == 64) {
+        // inference on 64-row tiles: fp16 copy of the centroids (scaled by a power of two from
+        // their largest magnitude), rows converted inside the kernel
+        CAT_CUDA(launch_absmax(C, (size_t)K * D, w.hscale, s));
+        CAT_CUDA(launch_half_scale(w.hscale, s));
+        CAT_CUDA(launch_to_half(C, (size_t)K * D, w.hscale, w.ch, s));
+        CAT_CUDA(launch_apply_h64(Y, N, D, K, w.ch, w.hscale, w.cnorm, labels, w.refine_rows, w.cand_rows, w.cand_list,
+                                  w.ctl, gamma, beta, out, s));
+        CAT_CUDA(launch_refine_both(Y, N, D, K, C, labels, w.cand_rows, w.cand_list, w.refine_rows, w.ctl, gamma,
+                                    beta, out, s));
+    } else if (use_tensor_path(N, D, K)) {
         if (!out && !row_norms_ready) CAT_CUDA(launch_row_norms(Y, N, D, w.ynorm2, s));
         if (Yh && !centroids_ready) CAT_CUDA(launch_to_half(C, (size_t)K * D, hscale, Ch, s));
         CAT_CUDA(launch_assign_tc(Y, N, D, K, C, w.cnorm, w.ynorm2, labels, w.refine_rows, w.cand_rows,
-                                  w.cand_list, w.ctl, gamma, beta, out, s, Yh, Ch, hscale));
+                                  w.cand_list, w.ctl, gamma, beta, out, s, Yh, Ch, hscale, fast));
         CAT_CUDA(launch_refine_both(Y, N, D, K, C, labels, w.cand_rows, w.cand_list, w.refine_rows, w.ctl, gamma,
                                     beta, out, s));
     } else {
-        CAT_CUDA(launch_assign(Y, N, D, K, C, w.cnorm, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
+        CAT_CUDA(launch_assign(Y, N, D, K, C, w.cnorm, labels, w.refine_rows, w.ctl, gamma, beta, out, s, fast));
         if (K > 1) CAT_CUDA(launch_refine(Y, N, D, K, C, labels, w.refine_rows, w.ctl, gamma, beta, out, s));
     }
     return CAT_OK;
@@ -243,6 +255,45 @@ cat_status_t cat_assign(const float *Yq, int64_t N, int32_t D, int32_t K, const 
                       reinterpret_cast<cudaStream_t>(stream));
 }
 
+cat_status_t cat_assign_scores(const float *Yq, int64_t N, int32_t D, int32_t K, const float *centroids,
+                               int32_t *labels_out, const cat_fast_scores_t *scores, int32_t flags,
+                               void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!Yq || !centroids || !labels_out) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (flags & ~CAT_ASSIGN_FP16_OPERANDS) return CAT_ERR_SHAPE;
+    if (!aligned16(Yq) || !aligned16(centroids) || !aligned16(labels_out)) return CAT_ERR_ALIGN;
+    FastOut fast;
+    if (scores) {
+        fast.best = scores->best;
+        fast.second = scores->second;
+        fast.bound = scores->bound;
+        fast.label = scores->label;
+    }
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (flags & CAT_ASSIGN_FP16_OPERANDS) {
+        if (!tc_half_supported(N, D, K) || N >= ((int64_t)1 << 30)) return CAT_ERR_UNSUPPORTED;
+        if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
+            return CAT_ERR_WORKSPACE;
+        FitWs w = carve_fit(workspace, N, D, K);
+        CAT_CUDA(launch_centroid_norms(centroids, D, K, w.a.cnorm, w.a.ctl, s, true));
+        CAT_CUDA(launch_half_shadow(Yq, N, D, w.a.ynorm2, w.hscale, w.yh, s));
+        CAT_CUDA(launch_to_half(centroids, (size_t)K * D, w.hscale, w.ch, s));
+        CAT_CUDA(launch_assign_tc(Yq, N, D, K, centroids, w.a.cnorm, w.a.ynorm2, labels_out, w.a.refine_rows,
+                                  w.a.cand_rows, w.a.cand_list, w.a.ctl, nullptr, nullptr, nullptr, s, w.yh, w.ch,
+                                  w.hscale, &fast));
+        CAT_CUDA(launch_refine_both(Yq, N, D, K, centroids, labels_out, w.a.cand_rows, w.a.cand_list, w.a.refine_rows,
+                                    w.a.ctl, nullptr, nullptr, nullptr, s));
+        return CAT_OK;
+    }
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_apply_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    AssignWs w = carve_assign(workspace, N, D, K);
+    return run_assign(Yq, N, D, K, centroids, labels_out, w, nullptr, nullptr, nullptr, s, false, true, nullptr, nullptr,
+                      nullptr, false, &fast);
+}
+
 cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t D, int32_t K,
                           int32_t iters, const float *init_centroids, float *centroids_out,
                           float *gamma_out, float *beta_out, int32_t *labels_out,
@@ -286,6 +337,7 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     // Lloyd rounds.  Two label buffers alternate so that a round sees the previous round's
     // labels and the final assignment lands in `labels`; the running per-cluster sums and
     // sizes start at zero with "no previous label" (-1) for every row.
+    const int diag_recorded = iters + 1 < CAT_DIAG_MAX_ROUNDS ? iters + 1 : CAT_DIAG_MAX_ROUNDS;
     int32_t *lab[2] = {labels, w.labels_prev};
     CAT_CUDA(cudaMemsetAsync(lab[(iters & 1) ^ 1], 0xFF, (size_t)N * sizeof(int32_t), s));
     CAT_CUDA(cudaMemsetAsync(w.sumQ, 0, KD * sizeof(double), s));
@@ -295,6 +347,9 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
         st = run_assign(Yq, N, D, K, C, cur, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale,
                         t > 0);
         if (st != CAT_OK) return st;
+        if (diag && t < CAT_DIAG_MAX_ROUNDS - 1)
+            CAT_CUDA(launch_fit_diag_round(Yq, N, D, K, C, cur, w.a.refine_rows, w.a.cand_rows, w.a.ctl, diag, t,
+                                           diag_recorded, s));
         st = run_delta_update(Yq, cur, prev, N, D, K, w, C, half, s);
         if (st != CAT_OK) return st;
     }
@@ -303,6 +358,9 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     st = run_assign(Yq, N, D, K, C, labels, w.a, nullptr, nullptr, nullptr, s, tc, false, Yh, w.ch, w.hscale,
                     iters > 0);
     if (st != CAT_OK) return st;
+    if (diag)
+        CAT_CUDA(launch_fit_diag_round(Yq, N, D, K, C, labels, w.a.refine_rows, w.a.cand_rows, w.a.ctl, diag,
+                                       diag_recorded - 1, diag_recorded, s));
     // The running sums follow the final labels too (without touching the centroids), which gives
     // the cluster means of Yq before the one sweep over Yq and Yfp that forms the centred moments
     // and the sums of Yfp.

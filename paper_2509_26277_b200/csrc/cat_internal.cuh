@@ -55,6 +55,14 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 #endif
 
 // ---------------------------------------------------------------- workspace layouts
+// Optional outputs of the fast pass (device pointers, each may be null): see cat_fast_scores_t.
+struct FastOut {
+    float *best = nullptr;
+    float *second = nullptr;
+    float *bound = nullptr;
+    int32_t *label = nullptr;
+};
+
 // Control block at the start of every workspace (device memory).
 struct Control {
     int32_t refine_count;        // rows queued for the exact fp64 pass by the current assignment
@@ -86,6 +94,8 @@ struct AssignWs {          // what assign/apply need
     float *ynorm2;         // [N] squared row norms (tensor-core labels-only path)
     int32_t *cand_rows;    // [N] rows queued with candidates
     uint64_t *cand_list;   // [N] their candidates, 4 x 16 bit
+    void *ch;              // [K*D] fp16 copy of the centroids (inference on fp16 operands)
+    float *hscale;         // [4] scale of that copy: {s_c, -2 / s_c, 2^-25 / s_c, -}
     size_t bytes;
 };
 AssignWs carve_assign(void *base, int64_t N, int D, int K);
@@ -121,7 +131,8 @@ cudaError_t launch_centroid_norms(const float *C, int D, int K, float *cnorm, Co
 // Fast fp32 scores + certainty test; optional fused affine epilogue.
 cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *C,
                           const float *cnorm, int32_t *labels, int32_t *refine_rows, Control *ctl,
-                          const float *gamma, const float *beta, float *out, cudaStream_t s);
+                          const float *gamma, const float *beta, float *out, cudaStream_t s,
+                          const FastOut *fast = nullptr);
 
 // Exact fp64 direct-form labels for the queued rows; optional affine output.
 cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *C,
@@ -130,16 +141,29 @@ cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *
 
 // Tensor-core (tcgen05, TF32) variant of launch_assign; ynorm2 is needed when out == nullptr.
 bool tc_supported(int64_t N, int D, int K);
-// Column-split form of the fused inference kernel: 0 = chosen by shape, 1 = never, 2 / 4 = that cluster size where it applies.
+// Form of the fused inference kernel on the tensor path: 0 = chosen by shape, 1 = TF32 row tiles
+// (128 rows per CTA), 2 / 4 = column split over that many CTAs where it applies, 64 = 64-row tiles
+// on fp16 operands made on the fly where that applies.
 void set_apply_column_split(int cs);
 int get_apply_column_split();
+int choose_apply_form(int64_t N, int D, int K);   // 1, 2, 4 or 64 for this shape under the current setting
+// 64-row-tile inference kernel on fp16 operands (cat_apply64.cu).  Ch = fp16(C * scale[0]) and
+// scale = {s_c, -2 / s_c, 2^-25 / s_c, -} come from launch_absmax + launch_half_scale + launch_to_half.
+bool apply_h64_supported(int64_t N, int D, int K);
+cudaError_t launch_absmax(const float *src, size_t n, float *scale, cudaStream_t s);   // scale[0] <- bits of max |src|
+cudaError_t launch_half_scale(float *scale, cudaStream_t s);                           // bits of the maximum -> the three scale words
+cudaError_t launch_apply_h64(const float *Y, int64_t N, int D, int K, const void *Ch, const float *scale,
+                             const float *cnorm, int32_t *labels, int32_t *refine_rows, int32_t *cand_rows,
+                             uint64_t *cand_list, Control *ctl, const float *gamma, const float *beta, float *out,
+                             cudaStream_t s);
 cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaStream_t s);
 // With Yh / Ch / scale (labels only): the fp16 copies of the rows and centroids are the MMA operands.
 cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,
                              const float *ynorm2, int32_t *labels, int32_t *refine_rows,
                              int32_t *cand_rows, uint64_t *cand_list, Control *ctl,
                              const float *gamma, const float *beta, float *out, cudaStream_t s,
-                             const void *Yh = nullptr, const void *Ch = nullptr, const float *scale = nullptr);
+                             const void *Yh = nullptr, const void *Ch = nullptr, const float *scale = nullptr,
+                             const FastOut *fast = nullptr);
 
 // One warp waits (at most limit_ms, clamped to 1 .. 1000) on a barrier that is never completed.
 cudaError_t launch_wait_selftest(Control *ctl, int limit_ms, cudaStream_t s);
@@ -202,6 +226,12 @@ cudaError_t launch_blend_params(const float *gamma, const float *beta, float alp
                                 float *gamma_b, float *beta_b, cudaStream_t s);
 cudaError_t launch_fit_diag(const Control *ctl, const int64_t *counts, int K, cat_fit_diag_t *diag,
                             cudaStream_t s);
+// Record of one assignment in diag (slot): objective against C for the given labels, rows that were
+// queued for the exact pass (the queues of the workspace as the exact pass left them), and how many
+// of those have their two nearest centroids within 1e-6 relative.  An extra pass over Y.
+cudaError_t launch_fit_diag_round(const float *Y, int64_t N, int D, int K, const float *C, const int32_t *labels,
+                                  const int32_t *refine_rows, const int32_t *cand_rows, const Control *ctl,
+                                  cat_fit_diag_t *diag, int slot, int recorded, cudaStream_t s);
 cudaError_t launch_reset_control(Control *ctl, cudaStream_t s);
 
 }  // namespace cat

@@ -111,6 +111,7 @@ struct AssignParams {
     int64_t N;
     int D;
     int K;
+    FastOut fast;
 };
 
 template <int BN>
@@ -323,6 +324,10 @@ __global__ void __launch_bounds__(A_THREADS) assign_kernel(AssignParams p)
             int k = sm.idx[tid];
             bool certain = (p.K == 1) || (gap > 2.f * e);
             p.labels[row] = k;
+            if (p.fast.best) p.fast.best[row] = sm.best[tid];
+            if (p.fast.second) p.fast.second[row] = sm.second[tid];
+            if (p.fast.bound) p.fast.bound[row] = e;
+            if (p.fast.label) p.fast.label[row] = k;
             if (certain) {
                 lab = k;
             } else {
@@ -404,9 +409,10 @@ static cudaError_t launch_assign_bn(const AssignParams &p, cudaStream_t s)
 
 cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *C,
                           const float *cnorm, int32_t *labels, int32_t *refine_rows, Control *ctl,
-                          const float *gamma, const float *beta, float *out, cudaStream_t s)
+                          const float *gamma, const float *beta, float *out, cudaStream_t s,
+                          const FastOut *fast)
 {
-    AssignParams p{Y, C, cnorm, labels, refine_rows, ctl, gamma, beta, out, N, D, K};
+    AssignParams p{Y, C, cnorm, labels, refine_rows, ctl, gamma, beta, out, N, D, K, fast ? *fast : FastOut{}};
     const bool vec = (D % 4 == 0);
     const bool affine = (out != nullptr);
     if (vec) return affine ? launch_assign_bn<true, true>(p, s) : launch_assign_bn<true, false>(p, s);
@@ -930,6 +936,98 @@ cudaError_t launch_fit_diag(const Control *ctl, const int64_t *counts, int K, ca
 {
     fit_diag_kernel<<<1, 32, 0, s>>>(ctl, counts, K, diag);
     count_launch();
+    return cudaGetLastError();
+}
+
+// ---- per-assignment diagnostics (only when the caller asks for them)
+
+// objective += sum over rows of ||y - c_label||^2 (fp64, one warp per row, one atomic per block)
+__global__ void __launch_bounds__(256) diag_objective_kernel(const float *__restrict__ Y, int64_t N, int D,
+                                                             const float *__restrict__ C,
+                                                             const int32_t *__restrict__ labels, double *objective)
+{
+    __shared__ double part[8];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    double acc = 0.0;
+    for (int64_t row = (int64_t)blockIdx.x * 8 + w; row < N; row += (int64_t)gridDim.x * 8) {
+        const float *y = Y + (size_t)row * D;
+        const float *c = C + (size_t)labels[row] * D;
+        double s = 0.0;
+        for (int j = lane; j < D; j += 32) {
+            const double d = (double)y[j] - (double)c[j];
+            s = fma(d, d, s);
+        }
+        acc += warp_sum(s);
+    }
+    if (lane == 0) part[w] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int q = 0; q < 8; ++q) t += part[q];
+        atomicAdd(objective, t);
+    }
+}
+
+// Rows of the two exact-pass queues whose two nearest centroids are within 1e-6 relative of each
+// other in squared distance (fp64 direct form over all K): one warp per queued row.
+__global__ void __launch_bounds__(256) diag_near_kernel(const float *__restrict__ Y, int64_t N, int D, int K,
+                                                        const float *__restrict__ C,
+                                                        const int32_t *__restrict__ refine_rows,
+                                                        const int32_t *__restrict__ cand_rows, const Control *ctl,
+                                                        long long *near_out)
+{
+    const int lane = threadIdx.x & 31;
+    int nref = ctl->refine_count, ncand = ctl->cand_count;
+    if ((int64_t)nref > N) nref = (int)N;
+    if ((int64_t)ncand > N) ncand = (int)N;
+    const int total = nref + ncand;
+    int found = 0;
+    for (int q = blockIdx.x * 8 + (threadIdx.x >> 5); q < total; q += gridDim.x * 8) {
+        const int64_t row = q < nref ? refine_rows[q] : cand_rows[q - nref];
+        if (row < 0 || row >= N) continue;
+        const float *y = Y + (size_t)row * D;
+        double best = CUDART_INF, second = CUDART_INF;
+        for (int k = 0; k < K; ++k) {
+            const float *c = C + (size_t)k * D;
+            double s = 0.0;
+            for (int j = lane; j < D; j += 32) {
+                const double d = (double)y[j] - (double)c[j];
+                s = fma(d, d, s);
+            }
+            s = warp_sum(s);
+            if (s < best) {
+                second = best;
+                best = s;
+            } else if (s < second) {
+                second = s;
+            }
+        }
+        if (K > 1 && (second - best) <= 1e-6 * second) ++found;
+    }
+    if (lane == 0 && found) atomicAdd(reinterpret_cast<unsigned long long *>(near_out), (unsigned long long)found);
+}
+
+__global__ void diag_round_begin_kernel(const Control *ctl, int64_t N, cat_fit_diag_t *diag, int slot, int recorded)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int64_t q = (int64_t)ctl->refine_count + (int64_t)ctl->cand_count;
+    diag->undecided_rows[slot] = q < N ? q : N;
+    diag->near_tie_rows[slot] = 0;
+    diag->objective[slot] = 0.0;
+    diag->assignments_recorded = recorded;
+}
+
+cudaError_t launch_fit_diag_round(const float *Y, int64_t N, int D, int K, const float *C, const int32_t *labels,
+                                  const int32_t *refine_rows, const int32_t *cand_rows, const Control *ctl,
+                                  cat_fit_diag_t *diag, int slot, int recorded, cudaStream_t s)
+{
+    diag_round_begin_kernel<<<1, 32, 0, s>>>(ctl, N, diag, slot, recorded);
+    int64_t blocks = (N + 7) / 8;
+    if (blocks > 1184) blocks = 1184;
+    diag_objective_kernel<<<(unsigned)blocks, 256, 0, s>>>(Y, N, D, C, labels, &diag->objective[slot]);
+    diag_near_kernel<<<(unsigned)blocks, 256, 0, s>>>(Y, N, D, K, C, refine_rows, cand_rows, ctl,
+                                                      reinterpret_cast<long long *>(&diag->near_tie_rows[slot]));
+    count_launch(3);
     return cudaGetLastError();
 }
 

@@ -1,7 +1,8 @@
 """Full-size workloads in the launch configuration bench.py times, checked on sampled
 outputs and on properties the oracle can verify at any size.
 
-Config 3 (200 704 x 64, K = 64) is small enough for the whole protocol.  Config 4
+Configs 0-2 (D = 1000; 1024, 50 000 and 50 000 apply rows) and config 3 (200 704 x 64, K = 64)
+are small enough for the whole protocol on every row.  Config 4
 (4 194 304 x 1024 apply, 262 144 x 1024 fit, K = 256) is checked by
   * apply: labels in range on every row; labels and outputs of a seeded row sample
     equal to the oracle's for the same parameters;
@@ -24,6 +25,33 @@ pytestmark = pytest.mark.gpu
 
 def host(t):
     return t.detach().cpu().numpy()
+
+
+@pytest.mark.parametrize("config", [0, 1, 2])
+@pytest.mark.parametrize("path", ["fp32", "tensor"])
+def test_linear_head_configs_full_size(config, path):
+    """The whole fit and the whole apply set (a row pitch of 4000 bytes, several tiles per CTA of the
+    persistent kernels), every row against the oracle, on both contraction paths."""
+    old = B.cat_get_tensor_core_min_k()
+    B.cat_set_tensor_core_min_k(1 << 30 if path == "fp32" else 1)
+    try:
+        w = W.make(config, device="cpu")
+        Yq, Yfp, Ya = w.Yq_fit.numpy(), w.Yfp_fit.numpy(), w.Yq_apply.numpy()
+        C, G, Bt, labels = B.cat_fit(w.Yq_fit.cuda(), w.Yfp_fit.cuda(), w.K, w.iters)
+        lab, best, second = O.assign(Yq, host(C))
+        labels_match(host(labels), lab, best, second, f"config {config} fit labels")
+        g_want, b_want = O.solve_gamma_beta(Yq, Yfp, host(labels), w.K)
+        close(host(G), g_want, f"config {config} gamma")
+        close(host(Bt), b_want, f"config {config} beta")
+        want, alab_want, best, second = O.apply(Ya, host(C), host(G), host(Bt))
+        out, alab = B.cat_apply(w.Yq_apply.cuda(), C, G, Bt, want_labels=True)
+        n_near, n_diff = labels_match(host(alab), alab_want, best, second, f"config {config} apply labels")
+        want2 = want if n_diff == 0 else O.affine_with_labels(Ya, host(alab), host(G), host(Bt))
+        err = close(host(out), want2, f"config {config} apply outputs")
+        print(f"config {config} ({path}): apply rows {len(Ya)}, near-tie rows {n_near} (label differs on {n_diff}), "
+              f"max |err| {err:.2e}")
+    finally:
+        B.cat_set_tensor_core_min_k(old)
 
 
 def test_config3_full_size():
@@ -87,14 +115,16 @@ def test_config4_full_size():
         y = w.Yq_apply[sl][:, cols].double()
         ref = (G[l][:, cols].double() * y + Bt[l][:, cols].double()).float()
         assert torch.equal(ref, out[sl][:, cols])
-    # the column-split form of the kernel gives the same labels and the same bits
+    # every form of the fused kernel gives the same labels and the same bits
     del y, ref, l
-    try:
-        B.cat_set_apply_column_split(2)
-        out2, alab2 = B.cat_apply(w.Yq_apply, C, G, Bt, want_labels=True)
-        torch.cuda.synchronize()
-    finally:
-        B.cat_set_apply_column_split(0)
-    assert torch.equal(alab2, alab)
-    assert torch.equal(out2, out)
+    for form in (1, 2, 64):
+        try:
+            B.cat_set_apply_column_split(form)
+            out2, alab2 = B.cat_apply(w.Yq_apply, C, G, Bt, want_labels=True)
+            torch.cuda.synchronize()
+        finally:
+            B.cat_set_apply_column_split(0)
+        assert torch.equal(alab2, alab), form
+        assert torch.equal(out2, out), form
+        del out2, alab2
     B.clear_workspaces()

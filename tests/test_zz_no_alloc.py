@@ -1,8 +1,8 @@
 """cat_assign_noalloc, the entry point for callers that cannot allocate device memory
 (it keeps its scratch in a fixed array inside the library).  Collected last on purpose.
 
-The check: through the C ABI, its labels equal cat_assign's on the same inputs, twice in a
-row -- the second call right after one that filled the shared scratch with a long queue of
+The check: through the C ABI, its labels equal cat_assign's (and the CPU oracle's) on the same
+inputs, twice in a row -- the second call right after one that filled the shared scratch with a long queue of
 exact-pass rows, so anything the first call left behind would show."""
 import ctypes
 
@@ -10,7 +10,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import cat_oracle as O
 from paper_2509_26277_b200 import binding as B
+from tests.parity import labels_match
 
 
 def test_noalloc_rejects_sizes_beyond_its_limits_on_the_host():
@@ -46,6 +48,9 @@ def test_noalloc_labels_equal_cat_assign_on_two_calls_in_a_row():
     torch.cuda.synchronize()
     assert torch.equal(got1, want1) and int(got1.max()) == 0
     assert torch.equal(got2, want2)
+    # and against the CPU oracle, which shares nothing with either entry point
+    lab, best, second = O.assign(Y2.cpu().numpy(), C2.cpu().numpy())
+    labels_match(got2.cpu().numpy(), lab, best, second, "cat_assign_noalloc labels")
     # and once more in the opposite order, at the row limit
     Y3 = torch.from_numpy(rng.normal(size=(B.NOALLOC_MAX_ROWS, 16)).astype(np.float32)).cuda()
     C3 = Y3[:200].clone()

@@ -17,7 +17,8 @@
  *     library allocates and frees nothing.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *     Calls only enqueue work: they return after launching, never synchronise,
- *     and are re-entrant for distinct workspaces.
+ *     and are re-entrant for distinct workspaces (the two
+ *     process-wide kernel selectors at the end of this header aside).
  *   - Return value: CAT_OK or an error code; on error nothing was enqueued
  *     (argument errors) or outputs are undefined (CAT_ERR_CUDA).  The library
  *     never throws, aborts or traps.
@@ -205,7 +206,8 @@ cat_status_t cat_assign_scores(const float *Yq, int64_t N, int32_t D, int32_t K,
 cat_status_t cat_assign_noalloc(const float *Yq, int64_t N, int32_t D, int32_t K,
                                 const float *centroids, int32_t *labels_out, void *stream);
 
-/* Per-cluster column sums of Y (fp64) and cluster sizes for given labels:
+/* Per-cluster column sums of Y (fp64) and cluster sizes for given labels (the sums behind the
+ * cluster means of the K-Means update, Section 4 Setup, and behind mu_LQ,k / mu_FP,k of Section 3.1):
  * sums_out [K, D] double, counts_out [K] int64.  Labels must lie in [0, K).
  * Rows are added in a fixed order: results are reproducible run to run.
  * Workspace: cat_fit_workspace_bytes(N, D, K). */
@@ -213,11 +215,13 @@ cat_status_t cat_cluster_sums(const float *Y, const int32_t *labels, int64_t N, 
                               int32_t K, double *sums_out, int64_t *counts_out,
                               void *workspace, size_t workspace_bytes, void *stream);
 
-/* c_k <- float(sums_k / counts_k) where counts_k > 0, else unchanged. */
+/* The centroid update of a K-Means round (Section 4 Setup: K-Means is the cluster model):
+ * c_k <- float(sums_k / counts_k) where counts_k > 0, else unchanged. */
 cat_status_t cat_centroids_from_sums(const double *sums, const int64_t *counts, int32_t D,
                                      int32_t K, float *centroids_inout, void *stream);
 
-/* Centred second moments for given labels and cluster means (fp64):
+/* Centred second moments for given labels and cluster means (fp64), the numerators of
+ * sigma^2_LQ,k and cov_LQ,FP,k of Section 3.1 (Algorithm 1, the Var and Mean of its loop body):
  *   var_out[k,j] = sum_{i in k} (q_ij - meanQ[k,j])^2
  *   cov_out[k,j] = sum_{i in k} (q_ij - meanQ[k,j]) (f_ij - meanF[k,j])
  * (sums, not yet divided by the cluster size).  Workspace as for cat_fit. */
@@ -285,21 +289,32 @@ cat_status_t cat_workspace_report(const void *workspace, void *stream, int64_t *
 cat_status_t cat_selftest_wait_timeout(void *workspace, size_t workspace_bytes, int32_t limit_ms, void *stream);
 
 /* Kernel selection for the distance contraction.  With K >= min_k (and D % 4 == 0,
- * K <= 256) the scores are formed on the tensor cores (tcgen05, TF32 operands, fp32
+ * K <= 256) the scores are formed on the tensor cores (tcgen05, TF32 or fp16 operands, fp32
  * accumulation); below it on the fp32 pipes.  Either way undecided rows are settled in
  * fp64, so the labels are the same.  Default 32: for smaller K the contraction is not
- * compute-limited.  Process-wide setting. */
+ * compute-limited.
+ * This and cat_set_apply_column_split are PROCESS-WIDE tuning and test hooks: they change
+ * which kernel every later call of every thread launches (never the results), and they are
+ * not meant to be flipped while other threads are inside the library. */
 void cat_set_tensor_core_min_k(int32_t min_k);
 int32_t cat_get_tensor_core_min_k(void);
 
-/* Kernel selection for the fused inference kernel (tensor-core path, D >= 128).  Two forms
- * compute the same thing: row tiles (a CTA pair shares 256 rows, each CTA all D columns of its
- * 128), and column split (the cs CTAs of a cluster share 128 rows, each staging D / cs columns;
- * the partial scores are summed through distributed shared memory).  The second keeps fewer
- * bytes in flight between a row's two reads, which pays once N x D no longer fits in L2.
- * cs = 0: chosen from the shape (default); 1: never split; 2 or 4: split over that many CTAs
- * wherever the shape allows it (D a multiple of 32 cs, K rounded up to 32 cs at most 256,
- * N > 128), row tiles elsewhere.  Other values count as 0.  Process-wide setting. */
+/* 1 if the tensor-core kernels can run in this process (the driver hands out the tensor-map
+ * encoder they need), 0 if not.  When it is 0 every call takes the fp32-pipe kernels, which
+ * give the same results about ten times slower for large K; callers that depend on the speed
+ * should check this once. */
+int32_t cat_tensor_path_available(void);
+
+/* Form of the fused inference kernel on the tensor-core path.  All forms compute the same thing
+ * (bit-identical outputs):
+ *   1   TF32 row tiles: a CTA pair shares 256 rows, each CTA all D columns of its 128;
+ *   2,4 column split: the CTAs of a cluster share 128 rows, each staging D / cs columns, partial
+ *       scores summed through distributed shared memory (needs D a multiple of 32 cs, K rounded
+ *       up to 32 cs at most 256, N > 128);
+ *   64  64-row tiles on fp16 operands converted inside the kernel (needs D >= 128, D % 8 == 0);
+ *   0   chosen from the shape (default).
+ * A form that the shape does not allow falls back to form 1.  Other values count as 0.
+ * Process-wide, see above. */
 void cat_set_apply_column_split(int32_t cs);
 int32_t cat_get_apply_column_split(void);
 

@@ -39,7 +39,7 @@ EXPORTS = [
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
     "cat_selftest_wait_timeout",
-    "cat_set_tensor_core_min_k", "cat_get_tensor_core_min_k",
+    "cat_set_tensor_core_min_k", "cat_get_tensor_core_min_k", "cat_tensor_path_available",
     "cat_set_apply_column_split", "cat_get_apply_column_split", "cat_status_string",
     "cat_last_cuda_error", "cat_version", "cat_kernel_launches",
 ]
@@ -110,6 +110,7 @@ def lib():
     L.cat_set_tensor_core_min_k.argtypes = [i32]
     L.cat_set_tensor_core_min_k.restype = None
     L.cat_get_tensor_core_min_k.restype = i32
+    L.cat_tensor_path_available.restype = i32
     L.cat_set_apply_column_split.argtypes = [i32]
     L.cat_set_apply_column_split.restype = None
     L.cat_get_apply_column_split.restype = i32
@@ -413,6 +414,10 @@ def cat_set_tensor_core_min_k(min_k: int) -> None:
 
 def cat_get_tensor_core_min_k() -> int:
     return int(lib().cat_get_tensor_core_min_k())
+
+
+def cat_tensor_path_available() -> bool:
+    return bool(lib().cat_tensor_path_available())
 
 
 def cat_set_apply_column_split(cs: int) -> None:

@@ -489,6 +489,8 @@ void cat_set_tensor_core_min_k(int32_t min_k)
 
 int32_t cat_get_tensor_core_min_k(void) { return g_tc_min_k.load(std::memory_order_relaxed); }
 
+int32_t cat_tensor_path_available(void) { return tc_supported(1, 4, 1) ? 1 : 0; }
+
 void cat_set_apply_column_split(int32_t cs) { set_apply_column_split((int)cs); }
 
 int32_t cat_get_apply_column_split(void) { return (int32_t)get_apply_column_split(); }

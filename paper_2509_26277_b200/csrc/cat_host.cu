@@ -3,6 +3,8 @@
 // cat_fit_host copies the fit set in, runs cat_fit and copies the model back.
 #include "cat_internal.cuh"
 
+#include <mutex>
+
 namespace cat {
 
 constexpr int H_SLOTS = 3;
@@ -61,6 +63,7 @@ struct HostPipe {
     cudaEvent_t in_ready[H_SLOTS], done[H_SLOTS], out_free[H_SLOTS], start = nullptr;
 };
 static HostPipe g_pipes[64];
+static std::mutex g_pipes_mu;   // first use on a device may come from several host threads at once
 
 static cudaError_t get_pipe(HostPipe **out)
 {
@@ -69,6 +72,7 @@ static cudaError_t get_pipe(HostPipe **out)
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     HostPipe &p = g_pipes[dev];
+    std::lock_guard<std::mutex> lock(g_pipes_mu);
     if (!p.ready) {
         if ((e = cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking)) != cudaSuccess) return e;
         if ((e = cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking)) != cudaSuccess) return e;

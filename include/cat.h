@@ -206,6 +206,42 @@ cat_status_t cat_assign_scores(const float *Yq, int64_t N, int32_t D, int32_t K,
 cat_status_t cat_assign_noalloc(const float *Yq, int64_t N, int32_t D, int32_t K,
                                 const float *centroids, int32_t *labels_out, void *stream);
 
+/*
+ * Row-sharded fitting (one shard of the rows per GPU).  K-Means (Section 4 Setup; Algorithm 1, the
+ * cluster model's fit) needs the rows only through per-cluster sums, so a Lloyd round splits into a
+ * local half -- assign this shard's rows, form what the round changed in the per-cluster sums -- and
+ * an update every rank repeats on the all-reduced changes.  The local half runs the same kernels as
+ * cat_fit (fp16 copy of the shard, exact pass for undecided rows, sums over the rows whose label
+ * changed), and the library issues no collective: the caller all-reduces between the calls.
+ *
+ *   cat_fit_shard_begin   once per fit: fp16 copy and norms of this shard's rows in the workspace;
+ *                         amax_out (device, 1 float) = largest magnitude of the shard.  The caller
+ *                         takes the maximum over all shards.
+ *   cat_fit_shard_round   round = 0, 1, 2, ... in order, on the same workspace: labels of the shard
+ *                         against `centroids`; delta_sums [K, D] double and delta_counts [K] int64
+ *                         receive, per cluster, (rows that entered) - (rows that left) since the
+ *                         previous round of this workspace (round 0: every row enters).  amax
+ *                         (device, 1 float) is the maximum over all shards from cat_fit_shard_begin.
+ *                         labels_out [N] may be NULL.  The caller sums the deltas over all shards.
+ *   cat_fit_shard_update  sums += delta_sums, counts += delta_counts, c_k = sums_k / counts_k where
+ *                         counts_k > 0 (a cluster with no rows keeps c_k); sums_inout / counts_inout
+ *                         are the caller's running totals, zero before round 0.
+ *
+ * With one shard the three calls reproduce cat_fit's Lloyd rounds bit for bit.  A further round call
+ * with the final centroids gives the final labels; the closed form then follows from
+ * cat_cluster_sums, cat_centred_moments and cat_solve_gamma_beta on all-reduced sums.
+ * Workspace: cat_fit_workspace_bytes(N, D, K) of the shard; N >= 1 (a shard may hold fewer than K rows).
+ */
+cat_status_t cat_fit_shard_begin(const float *Yq, int64_t N, int32_t D, int32_t K, float *amax_out,
+                                 void *workspace, size_t workspace_bytes, void *stream);
+cat_status_t cat_fit_shard_round(const float *Yq, int64_t N, int32_t D, int32_t K, int32_t round,
+                                 const float *centroids, const float *amax, double *delta_sums,
+                                 int64_t *delta_counts, int32_t *labels_out,
+                                 void *workspace, size_t workspace_bytes, void *stream);
+cat_status_t cat_fit_shard_update(const double *delta_sums, const int64_t *delta_counts, int32_t D,
+                                  int32_t K, double *sums_inout, int64_t *counts_inout,
+                                  float *centroids_inout, void *stream);
+
 /* Per-cluster column sums of Y (fp64) and cluster sizes for given labels (the sums behind the
  * cluster means of the K-Means update, Section 4 Setup, and behind mu_LQ,k / mu_FP,k of Section 3.1):
  * sums_out [K, D] double, counts_out [K] int64.  Labels must lie in [0, K).

@@ -35,6 +35,7 @@ class _FastScores(ctypes.Structure):       # cat_fast_scores_t
 EXPORTS = [
     "cat_fit_workspace_bytes", "cat_fit", "cat_fit_from", "cat_apply_workspace_bytes",
     "cat_apply", "cat_apply_blend", "cat_assign", "cat_assign_scores", "cat_assign_noalloc", "cat_cluster_sums",
+    "cat_fit_shard_begin", "cat_fit_shard_round", "cat_fit_shard_update",
     "cat_centroids_from_sums",
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
@@ -93,6 +94,11 @@ def lib():
     L.cat_assign_scores.restype = ctypes.c_int
     L.cat_assign_noalloc.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     L.cat_assign_noalloc.restype = ctypes.c_int
+    L.cat_fit_shard_begin.argtypes = [vp, i64, i32, i32, vp, vp, sz, vp]
+    L.cat_fit_shard_round.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.cat_fit_shard_update.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    for name in ("cat_fit_shard_begin", "cat_fit_shard_round", "cat_fit_shard_update"):
+        getattr(L, name).restype = ctypes.c_int
     L.cat_cluster_sums.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, sz, vp]
     L.cat_centroids_from_sums.argtypes = [vp, vp, i32, i32, vp, vp]
     L.cat_centred_moments.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, vp, vp, sz, vp]
@@ -310,6 +316,28 @@ def cat_assign_noalloc(Yq, centroids, labels_out):
                                   _dev(labels_out, torch.int32, (N,), "labels_out"), _stream())
     _check(st, "cat_assign_noalloc")
     return labels_out
+
+
+def cat_fit_shard_begin(Yq, K: int, amax_out, ws):
+    N, D = Yq.shape
+    _check(lib().cat_fit_shard_begin(_dev(Yq, torch.float32, None, "Yq"), N, D, K, _dev(amax_out, torch.float32, (1,)),
+                                     ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream()), "cat_fit_shard_begin")
+
+
+def cat_fit_shard_round(Yq, K: int, rnd: int, centroids, amax, delta_sums, delta_counts, labels_out, ws):
+    N, D = Yq.shape
+    _check(lib().cat_fit_shard_round(_dev(Yq, torch.float32, None, "Yq"), N, D, K, int(rnd),
+                                     _dev(centroids, torch.float32, (K, D), "centroids"), _dev(amax, torch.float32, (1,)),
+                                     _dev(delta_sums, torch.float64, (K, D)), _dev(delta_counts, torch.int64, (K,)),
+                                     _dev(labels_out, torch.int32, (N,)),
+                                     ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream()), "cat_fit_shard_round")
+
+
+def cat_fit_shard_update(delta_sums, delta_counts, sums, counts, centroids):
+    K, D = centroids.shape
+    _check(lib().cat_fit_shard_update(_dev(delta_sums, torch.float64, (K, D)), _dev(delta_counts, torch.int64, (K,)),
+                                      D, K, _dev(sums, torch.float64, (K, D)), _dev(counts, torch.int64, (K,)),
+                                      _dev(centroids, torch.float32, (K, D)), _stream()), "cat_fit_shard_update")
 
 
 def cat_cluster_sums(Y, labels, K: int, ws=None):

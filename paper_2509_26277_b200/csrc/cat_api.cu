@@ -394,6 +394,88 @@ cat_status_t cat_fit(const float *Yq, const float *Yfp, int64_t N, int32_t D, in
                         labels_out, nullptr, workspace, workspace_bytes, stream);
 }
 
+// ---- row-sharded fitting: the local half of a Lloyd round and the replicated update
+
+cat_status_t cat_fit_shard_begin(const float *Yq, int64_t N, int32_t D, int32_t K, float *amax_out,
+                                 void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!Yq || !amax_out) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (N >= ((int64_t)1 << 30)) return CAT_ERR_UNSUPPORTED;
+    if (!aligned16(Yq)) return CAT_ERR_ALIGN;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    FitWs w = carve_fit(workspace, N, D, K);
+    CAT_CUDA(launch_reset_control(w.a.ctl, s));
+    CAT_CUDA(cudaMemsetAsync(w.hscale, 0, 4 * sizeof(float), s));
+    const bool tc = use_tensor_path(N, D, K);
+    if (tc && tc_half_supported(N, D, K))
+        CAT_CUDA(launch_half_shadow(Yq, N, D, w.a.ynorm2, w.hscale, w.yh, s, false));
+    else if (tc)
+        CAT_CUDA(launch_row_norms(Yq, N, D, w.a.ynorm2, s));
+    // (the bit pattern of a non-negative float is the float itself)
+    CAT_CUDA(cudaMemcpyAsync(amax_out, w.hscale, sizeof(float), cudaMemcpyDeviceToDevice, s));
+    // round 0 sees "no previous label" for every row
+    CAT_CUDA(cudaMemsetAsync(w.labels_prev, 0xFF, (size_t)N * sizeof(int32_t), s));
+    return CAT_OK;
+}
+
+cat_status_t cat_fit_shard_round(const float *Yq, int64_t N, int32_t D, int32_t K, int32_t round,
+                                 const float *centroids, const float *amax, double *delta_sums,
+                                 int64_t *delta_counts, int32_t *labels_out, void *workspace,
+                                 size_t workspace_bytes, void *stream)
+{
+    if (!Yq || !centroids || !amax || !delta_sums || !delta_counts) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (round < 0) return CAT_ERR_SHAPE;
+    if (N >= ((int64_t)1 << 30)) return CAT_ERR_UNSUPPORTED;
+    if (!aligned16(Yq) || !aligned16(centroids) || !aligned16(delta_sums) || !aligned16(delta_counts) ||
+        (labels_out && !aligned16(labels_out)))
+        return CAT_ERR_ALIGN;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_fit_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    FitWs w = carve_fit(workspace, N, D, K);
+    const bool tc = use_tensor_path(N, D, K);
+    const bool half = tc && tc_half_supported(N, D, K);
+    // the two label buffers of the workspace alternate; round 0 reads the all -1 buffer cat_fit_shard_begin left
+    int32_t *cur = (round & 1) ? w.labels_prev : w.a.labels;
+    int32_t *prev = (round & 1) ? w.a.labels : w.labels_prev;
+    if (half) {
+        CAT_CUDA(cudaMemcpyAsync(w.hscale, amax, sizeof(float), cudaMemcpyDeviceToDevice, s));
+        CAT_CUDA(launch_half_scale(w.hscale, s));
+    }
+    st = run_assign(Yq, N, D, K, centroids, cur, w.a, nullptr, nullptr, nullptr, s, tc, false, half ? w.yh : nullptr,
+                    w.ch, w.hscale, false);
+    if (st != CAT_OK) return st;
+    const size_t KD = (size_t)K * D;
+    CAT_CUDA(cudaMemsetAsync(delta_sums, 0, KD * sizeof(double), s));
+    CAT_CUDA(cudaMemsetAsync(delta_counts, 0, (size_t)K * sizeof(int64_t), s));
+    SegGeom g = seg_geometry(2 * N, D, 2 * K);
+    CAT_CUDA(launch_label_sort(cur, prev, N, K, g, w.blk_hist, w.key_total, delta_counts, w.cluster_start,
+                               w.seg_start, w.order, s));
+    CAT_CUDA(launch_segment_sums(0, Yq, nullptr, w.order, w.cluster_start, w.seg_start, nullptr, nullptr, D, 2 * K, g,
+                                 w.segpart, s));
+    CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, nullptr, D, K, true, delta_sums, nullptr, nullptr, s));
+    if (labels_out)
+        CAT_CUDA(cudaMemcpyAsync(labels_out, cur, (size_t)N * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
+    return CAT_OK;
+}
+
+cat_status_t cat_fit_shard_update(const double *delta_sums, const int64_t *delta_counts, int32_t D, int32_t K,
+                                  double *sums_inout, int64_t *counts_inout, float *centroids_inout, void *stream)
+{
+    if (!delta_sums || !delta_counts || !sums_inout || !counts_inout || !centroids_inout) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(K, D, K, false);
+    if (st != CAT_OK) return st;
+    CAT_CUDA(launch_shard_update(delta_sums, delta_counts, D, K, sums_inout, counts_inout, centroids_inout,
+                                 reinterpret_cast<cudaStream_t>(stream)));
+    return CAT_OK;
+}
+
 cat_status_t cat_cluster_sums(const float *Y, const int32_t *labels, int64_t N, int32_t D,
                               int32_t K, double *sums_out, int64_t *counts_out, void *workspace,
                               size_t workspace_bytes, void *stream)

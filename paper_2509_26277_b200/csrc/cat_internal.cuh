@@ -172,8 +172,10 @@ cudaError_t launch_wait_selftest(Control *ctl, int limit_ms, cudaStream_t s);
 // power-of-two scales, Yh[i] = fp16(Y[i] * scale_i), and scale[4 + N] = {centroid scale s_c from the
 // largest magnitude, -2 / s_c, 2^-25 / s_c, unused, then 1 / scale_i for every row}.  Needs D % 8 == 0.
 bool tc_half_supported(int64_t N, int D, int K);
+// finish_scale = false leaves the bits of the largest magnitude in scale[0] (launch_half_scale turns them
+// into the three scale words later, e.g. once the maximum over several shards is known).
 cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, float *scale, void *Yh,
-                               cudaStream_t s);
+                               cudaStream_t s, bool finish_scale = true);
 // dst = fp16(src * scale[0]) for n elements (n % 4 == 0)
 cudaError_t launch_to_half(const float *src, size_t n, const float *scale, void *dst, cudaStream_t s);
 
@@ -217,6 +219,9 @@ cudaError_t launch_centroid_update(const double *part, const int32_t *seg_start,
 
 cudaError_t launch_centroids_from_sums(const double *sums, const int64_t *counts, int D, int K,
                                        float *C, cudaStream_t s);
+// sums += delta_sums, counts += delta_counts, C = float(sums / counts) where counts > 0
+cudaError_t launch_shard_update(const double *delta_sums, const int64_t *delta_counts, int D, int K, double *sums,
+                                int64_t *counts, float *C, cudaStream_t s);
 cudaError_t launch_means_from_sums(const double *sums, const int64_t *counts, int D, int K,
                                    double *mean, cudaStream_t s);
 cudaError_t launch_solve(const double *sumQ, const double *sumF, const double *var,

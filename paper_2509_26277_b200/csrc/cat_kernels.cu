@@ -840,6 +840,35 @@ cudaError_t launch_centroids_from_sums(const double *sums, const int64_t *counts
     return cudaGetLastError();
 }
 
+// one block per cluster: the cluster's size first (by thread 0, before anyone reads it), then its columns
+__global__ void shard_update_kernel(const double *__restrict__ dsums, const int64_t *__restrict__ dcounts, int D,
+                                    double *__restrict__ sums, int64_t *__restrict__ counts, float *__restrict__ C)
+{
+    __shared__ long long n_s;
+    const int k = blockIdx.x;
+    if (threadIdx.x == 0) {
+        const long long n = (long long)counts[k] + (long long)dcounts[k];
+        counts[k] = n;
+        n_s = n;
+    }
+    __syncthreads();
+    const long long n = n_s;
+    for (int j = threadIdx.x; j < D; j += blockDim.x) {
+        const size_t e = (size_t)k * D + j;
+        const double a = sums[e] + dsums[e];
+        sums[e] = a;
+        if (n > 0) C[e] = (float)(a / (double)n);
+    }
+}
+
+cudaError_t launch_shard_update(const double *delta_sums, const int64_t *delta_counts, int D, int K, double *sums,
+                                int64_t *counts, float *C, cudaStream_t s)
+{
+    shard_update_kernel<<<K, 256, 0, s>>>(delta_sums, delta_counts, D, sums, counts, C);
+    count_launch();
+    return cudaGetLastError();
+}
+
 __global__ void means_from_sums_kernel(const double *__restrict__ sums,
                                        const int64_t *__restrict__ counts, int D, size_t KD,
                                        double *__restrict__ mean)

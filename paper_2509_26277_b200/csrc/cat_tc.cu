@@ -1099,7 +1099,7 @@ cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaS
 }
 
 cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, float *scale, void *Yh,
-                               cudaStream_t s)
+                               cudaStream_t s, bool finish_scale)
 {
     float *rinv = scale + 4;
     cudaError_t e = cudaMemsetAsync(scale, 0, 4 * sizeof(float), s);
@@ -1111,8 +1111,8 @@ cudaError_t launch_half_shadow(const float *Y, int64_t N, int D, float *ynorm2, 
     if (blocks > cap) blocks = cap;
     half_shadow_kernel<<<(unsigned)blocks, 256, 0, s>>>(Y, N, D, G, ynorm2, rinv, reinterpret_cast<unsigned int *>(scale),
                                                         reinterpret_cast<__half *>(Yh));
-    half_scale_kernel<<<1, 32, 0, s>>>(scale);
-    count_launch(2);
+    if (finish_scale) half_scale_kernel<<<1, 32, 0, s>>>(scale);
+    count_launch(finish_scale ? 2 : 1);
     return cudaGetLastError();
 }
 

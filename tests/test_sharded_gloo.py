@@ -17,19 +17,37 @@ from paper_2509_26277_b200 import sharded
 class CpuStandIn:
     """Per-rank steps for the test: the oracle's assignment, numpy fp64 sums."""
 
-    def assign(self, Yq, C):
-        return torch.from_numpy(O.assign(Yq.numpy(), C.numpy())[0])
+    def begin(self, Yq, K):
+        self.K = K
+        self.prev = None
+        return Yq.abs().max().reshape(1).float()
+
+    def round(self, Yq, rnd, C, amax):
+        """Labels from the oracle; what changed in the per-cluster sums since the previous round."""
+        labels = O.assign(Yq.numpy(), C.numpy())[0]
+        y = Yq.numpy().astype(np.float64)
+        dsums = np.zeros((self.K, y.shape[1]), np.float64)
+        dcounts = np.zeros(self.K, np.int64)
+        moved = np.ones(len(y), bool) if self.prev is None else labels != self.prev
+        np.add.at(dsums, labels[moved], y[moved])
+        np.add.at(dcounts, labels[moved], 1)
+        if self.prev is not None:
+            np.add.at(dsums, self.prev[moved], -y[moved])
+            np.add.at(dcounts, self.prev[moved], -1)
+        self.prev = labels
+        return torch.from_numpy(dsums), torch.from_numpy(dcounts), torch.from_numpy(labels)
+
+    def update(self, dsums, dcounts, sums, counts, C):
+        sums += dsums
+        counts += dcounts
+        m = counts > 0
+        C[m] = (sums[m] / counts[m].double()[:, None]).float()
 
     def cluster_sums(self, Y, labels, K):
         sums = np.zeros((K, Y.shape[1]), np.float64)
         np.add.at(sums, labels.numpy(), Y.numpy().astype(np.float64))
         counts = np.bincount(labels.numpy(), minlength=K).astype(np.int64)
         return torch.from_numpy(sums), torch.from_numpy(counts)
-
-    def centroids_from_sums(self, sums, counts, C):
-        m = counts > 0
-        C[m] = (sums[m] / counts[m].double()[:, None]).float()
-        return C
 
     def centred_moments(self, Yq, Yfp, labels, meanQ, meanF):
         l = labels.numpy()
@@ -75,6 +93,22 @@ def _worker(rank, world, port, q):
                                               5, 6, backend=CpuStandIn())
         out = sharded.apply_sharded(torch.from_numpy(Yq[lo:hi]), C, g, b, backend=CpuStandIn())
         q.put((rank, lo, hi, C.numpy(), g.numpy(), b.numpy(), labels.numpy(), out.numpy()))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def _worker_uneven(rank, world, port, q):
+    """Rank 1 holds no rows at all: it must pass through every collective with zeros."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        Yq, Yfp = _data()
+        lo, hi = (0, len(Yq)) if rank == 0 else (len(Yq), len(Yq))
+        C, g, b, labels = sharded.fit_sharded(torch.from_numpy(Yq[lo:hi]), torch.from_numpy(Yfp[lo:hi]),
+                                              5, 4, backend=CpuStandIn())
+        q.put((rank, C.numpy(), g.numpy(), b.numpy(), labels.numpy()))
         dist.barrier()
     finally:
         dist.destroy_process_group()
@@ -127,3 +161,27 @@ def test_two_rank_gloo_fit_equals_single_process_oracle():
     # both ranks hold bit-identical models
     for a, b_ in zip(results[0][3:6], results[1][3:6]):
         assert np.array_equal(a, b_)
+
+
+@pytest.mark.timeout(300)
+def test_a_rank_without_rows_takes_part_with_zeros():
+    world = 2
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker_uneven, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted([q.get(timeout=240) for _ in range(world)], key=lambda x: x[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    Yq, Yfp = _data()
+    ora = O.fit(Yq, Yfp, 5, 4)
+    for rank, C, g, b, labels in results:
+        np.testing.assert_allclose(C, ora.centroids, rtol=1e-6, atol=1e-6)
+        np.testing.assert_allclose(g, ora.gamma, rtol=1e-5, atol=1e-6)
+        np.testing.assert_allclose(b, ora.beta, rtol=1e-5, atol=1e-6)
+    assert np.array_equal(results[0][4], ora.labels) and len(results[1][4]) == 0

@@ -34,7 +34,7 @@ from paper_2509_26277_b200 import workloads as W
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the fused inference kernel per row at D = 1024, K = 256
 # (the ncu capture summarised in profiles/; None while no capture of the current kernel exists)
-APPLY_DRAM_BYTES_PER_ROW = None
+APPLY_DRAM_BYTES_PER_ROW = 10658.0
 
 METRIC = "CAT rows/s through the hot path (fit row-passes + apply rows); see apply_rows_per_s, fit_s_per_lloyd_iter"
 UNIT = "rows/s"

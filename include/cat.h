@@ -275,6 +275,54 @@ cat_status_t cat_solve_gamma_beta(const double *sumQ, const double *sumF,
                                   const int64_t *counts, int32_t D, int32_t K,
                                   float *gamma_out, float *beta_out, void *stream);
 
+/* ---- PCA front-end ------------------------------------------------------ */
+
+/*
+ * Section 3.1 clusters the LQ outputs after reducing them with PCA ("PCA is only used to obtain
+ * clusters": gamma and beta stay in the original D-dimensional space).  Algorithm 1 step 1 fits
+ * the projection on the LQ outputs of the fit set, Algorithm 2 step 1 applies it at inference.
+ *
+ * cat_pca_fit: column means of Yq [N, D] -> mean_out [D]; covariance of the centred rows in fp64
+ * (1 / (N - 1)); its eigen-decomposition by one-sided Jacobi rotations in fp64 on the device; the p
+ * directions of largest variance -> components_out [p, D] (rows, unit length, decreasing variance;
+ * the sign of a row is fixed so that its entry of largest magnitude is positive); their variances
+ * -> eigenvalues_out [p] double, may be NULL.  Deterministic.  N >= 2, 1 <= p <= D,
+ * D <= CAT_PCA_MAX_D, p <= CAT_PCA_MAX_P.  Directions whose variances coincide are determined
+ * only up to a rotation among themselves.
+ * cat_pca_project: Z_out [N, p] = (Y - mean) components^T, fp64 accumulation, fp32 result.
+ * cat_affine_with_labels: Y_out_i = gamma_l * Yq_i + beta_l for given cluster ids l = labels[i]
+ * (Algorithm 2, the loop over the samples with alpha = 1); a label outside [0, K) copies the row.
+ */
+#define CAT_PCA_MAX_D 4096
+#define CAT_PCA_MAX_P 512
+size_t cat_pca_workspace_bytes(int64_t N, int32_t D, int32_t p);
+cat_status_t cat_pca_fit(const float *Yq, int64_t N, int32_t D, int32_t p, float *mean_out,
+                         float *components_out, double *eigenvalues_out,
+                         void *workspace, size_t workspace_bytes, void *stream);
+cat_status_t cat_pca_project(const float *Y, int64_t N, int32_t D, int32_t p, const float *mean,
+                             const float *components, float *Z_out, void *stream);
+cat_status_t cat_affine_with_labels(const float *Yq, int64_t N, int32_t D, int32_t K,
+                                    const int32_t *labels, const float *gamma, const float *beta,
+                                    float *Y_out, void *stream);
+
+/*
+ * Algorithm 1 as printed: PCA on Yq, K-Means on the reduced rows (first K reduced rows as the
+ * start, `iters` Lloyd rounds, a final assignment), then per cluster the closed-form gamma / beta
+ * from the original Yq, Yfp.  centroids_out is [K, p]; gamma_out, beta_out are [K, D].
+ * Algorithm 2 as printed (alpha = 1): project, nearest centroid in the reduced space, affine
+ * correction in the original space.
+ */
+size_t cat_fit_pca_workspace_bytes(int64_t N, int32_t D, int32_t K, int32_t p);
+cat_status_t cat_fit_pca(const float *Yq, const float *Yfp, int64_t N, int32_t D, int32_t K,
+                         int32_t iters, int32_t p, float *mean_out, float *components_out,
+                         float *centroids_out, float *gamma_out, float *beta_out, int32_t *labels_out,
+                         void *workspace, size_t workspace_bytes, void *stream);
+size_t cat_apply_pca_workspace_bytes(int64_t N, int32_t D, int32_t K, int32_t p);
+cat_status_t cat_apply_pca(const float *Yq, int64_t N, int32_t D, int32_t K, int32_t p,
+                           const float *mean, const float *components, const float *centroids,
+                           const float *gamma, const float *beta, float *Y_out, int32_t *labels_out,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- host-buffer entry points (end-to-end use) ------------------------- */
 
 /*

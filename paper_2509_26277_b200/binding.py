@@ -36,6 +36,8 @@ EXPORTS = [
     "cat_fit_workspace_bytes", "cat_fit", "cat_fit_from", "cat_apply_workspace_bytes",
     "cat_apply", "cat_apply_blend", "cat_assign", "cat_assign_scores", "cat_assign_noalloc", "cat_cluster_sums",
     "cat_fit_shard_begin", "cat_fit_shard_round", "cat_fit_shard_update",
+    "cat_pca_workspace_bytes", "cat_pca_fit", "cat_pca_project", "cat_affine_with_labels",
+    "cat_fit_pca_workspace_bytes", "cat_fit_pca", "cat_apply_pca_workspace_bytes", "cat_apply_pca",
     "cat_centroids_from_sums",
     "cat_centred_moments", "cat_solve_gamma_beta", "cat_apply_host_workspace_bytes",
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
@@ -98,6 +100,19 @@ def lib():
     L.cat_fit_shard_round.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     L.cat_fit_shard_update.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     for name in ("cat_fit_shard_begin", "cat_fit_shard_round", "cat_fit_shard_update"):
+        getattr(L, name).restype = ctypes.c_int
+    L.cat_pca_workspace_bytes.argtypes = [i64, i32, i32]
+    L.cat_pca_workspace_bytes.restype = sz
+    L.cat_fit_pca_workspace_bytes.argtypes = [i64, i32, i32, i32]
+    L.cat_fit_pca_workspace_bytes.restype = sz
+    L.cat_apply_pca_workspace_bytes.argtypes = [i64, i32, i32, i32]
+    L.cat_apply_pca_workspace_bytes.restype = sz
+    L.cat_pca_fit.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.cat_pca_project.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp]
+    L.cat_affine_with_labels.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp]
+    L.cat_fit_pca.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.cat_apply_pca.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    for name in ("cat_pca_fit", "cat_pca_project", "cat_affine_with_labels", "cat_fit_pca", "cat_apply_pca"):
         getattr(L, name).restype = ctypes.c_int
     L.cat_cluster_sums.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, sz, vp]
     L.cat_centroids_from_sums.argtypes = [vp, vp, i32, i32, vp, vp]
@@ -338,6 +353,82 @@ def cat_fit_shard_update(delta_sums, delta_counts, sums, counts, centroids):
     _check(lib().cat_fit_shard_update(_dev(delta_sums, torch.float64, (K, D)), _dev(delta_counts, torch.int64, (K,)),
                                       D, K, _dev(sums, torch.float64, (K, D)), _dev(counts, torch.int64, (K,)),
                                       _dev(centroids, torch.float32, (K, D)), _stream()), "cat_fit_shard_update")
+
+
+def _scratch(nbytes: int, device, where: str):
+    if nbytes == 0:
+        raise CatError(7, where + " workspace query")
+    return torch.empty(int(nbytes), dtype=torch.uint8, device=device)
+
+
+def cat_pca_fit(Yq, p: int, want_eigenvalues=False):
+    """Returns (mean [D], components [p, D][, eigenvalues float64 [p]])."""
+    N, D = Yq.shape
+    dev = Yq.device
+    mean = torch.empty((D,), dtype=torch.float32, device=dev)
+    comps = torch.empty((p, D), dtype=torch.float32, device=dev)
+    eig = torch.empty((p,), dtype=torch.float64, device=dev) if want_eigenvalues else None
+    ws = _scratch(lib().cat_pca_workspace_bytes(N, D, p), dev, "cat_pca_fit")
+    _check(lib().cat_pca_fit(_dev(Yq, torch.float32, None, "Yq"), N, D, p, _dev(mean, torch.float32),
+                             _dev(comps, torch.float32), _dev(eig, torch.float64),
+                             ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream()), "cat_pca_fit")
+    return (mean, comps, eig) if want_eigenvalues else (mean, comps)
+
+
+def cat_pca_project(Y, mean, comps):
+    N, D = Y.shape
+    p = comps.shape[0]
+    Z = torch.empty((N, p), dtype=torch.float32, device=Y.device)
+    _check(lib().cat_pca_project(_dev(Y, torch.float32, None, "Y"), N, D, p, _dev(mean, torch.float32, (D,), "mean"),
+                                 _dev(comps, torch.float32, (p, D), "components"), _dev(Z, torch.float32), _stream()),
+           "cat_pca_project")
+    return Z
+
+
+def cat_affine_with_labels(Yq, labels, gamma, beta, out=None):
+    N, D = Yq.shape
+    K = gamma.shape[0]
+    if out is None:
+        out = torch.empty_like(Yq)
+    _check(lib().cat_affine_with_labels(_dev(Yq, torch.float32, None, "Yq"), N, D, K, _dev(labels, torch.int32, (N,), "labels"),
+                                        _dev(gamma, torch.float32, (K, D), "gamma"), _dev(beta, torch.float32, (K, D), "beta"),
+                                        _dev(out, torch.float32, (N, D), "out"), _stream()), "cat_affine_with_labels")
+    return out
+
+
+def cat_fit_pca(Yq, Yfp, K: int, iters: int, p: int):
+    """Returns dict(mean, comps, centroids [K, p], gamma, beta [K, D], labels)."""
+    N, D = Yq.shape
+    dev = Yq.device
+    r = dict(mean=torch.empty((D,), dtype=torch.float32, device=dev),
+             comps=torch.empty((p, D), dtype=torch.float32, device=dev),
+             centroids=torch.empty((K, p), dtype=torch.float32, device=dev),
+             gamma=torch.empty((K, D), dtype=torch.float32, device=dev),
+             beta=torch.empty((K, D), dtype=torch.float32, device=dev),
+             labels=torch.empty((N,), dtype=torch.int32, device=dev))
+    ws = _scratch(lib().cat_fit_pca_workspace_bytes(N, D, K, p), dev, "cat_fit_pca")
+    _check(lib().cat_fit_pca(_dev(Yq, torch.float32, None, "Yq"), _dev(Yfp, torch.float32, (N, D), "Yfp"), N, D, K, iters, p,
+                             _dev(r["mean"], torch.float32), _dev(r["comps"], torch.float32),
+                             _dev(r["centroids"], torch.float32), _dev(r["gamma"], torch.float32),
+                             _dev(r["beta"], torch.float32), _dev(r["labels"], torch.int32),
+                             ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream()), "cat_fit_pca")
+    return r
+
+
+def cat_apply_pca(Yq, mean, comps, centroids, gamma, beta, out=None, want_labels=False):
+    N, D = Yq.shape
+    K, p = centroids.shape
+    dev = Yq.device
+    if out is None:
+        out = torch.empty_like(Yq)
+    labels = torch.empty((N,), dtype=torch.int32, device=dev) if want_labels else None
+    ws = _scratch(lib().cat_apply_pca_workspace_bytes(N, D, K, p), dev, "cat_apply_pca")
+    _check(lib().cat_apply_pca(_dev(Yq, torch.float32, None, "Yq"), N, D, K, p, _dev(mean, torch.float32, (D,)),
+                               _dev(comps, torch.float32, (p, D)), _dev(centroids, torch.float32, (K, p)),
+                               _dev(gamma, torch.float32, (K, D)), _dev(beta, torch.float32, (K, D)),
+                               _dev(out, torch.float32, (N, D)), _dev(labels, torch.int32),
+                               ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream()), "cat_apply_pca")
+    return (out, labels) if want_labels else out
 
 
 def cat_cluster_sums(Y, labels, K: int, ws=None):

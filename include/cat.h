@@ -138,6 +138,20 @@ cat_status_t cat_apply_blend(const float *Yq, int64_t N, int32_t D, int32_t K,
                              float alpha, float *Y_out, int32_t *labels_out,
                              void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * cat_apply with a bf16 result: Y_out_bf16 [N, D] receives bf16(gamma_l * Yq_i + beta_l), the fp32
+ * fused multiply-add of cat_apply rounded to nearest even (Algorithm 2 with alpha = 1; Section 3.1
+ * notes that the correction suits low-precision deployment, without fixing a format).  The labels
+ * are exact as in cat_apply.  Halves the bytes written.  For shapes the 64-row-tile kernel takes
+ * (K >= the tensor-core threshold, K <= 256, D >= 128, D % 8 == 0, N > 64) assignment and correction
+ * are fused; other shapes run the assignment, then one pass that reads the rows again.
+ * Workspace: cat_apply_workspace_bytes(N, D, K).
+ */
+cat_status_t cat_apply_bf16(const float *Yq, int64_t N, int32_t D, int32_t K,
+                            const float *centroids, const float *gamma, const float *beta,
+                            void *Y_out_bf16, int32_t *labels_out,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- step-level entry points (the same kernels cat_fit chains; used for
  *      row-sharded multi-GPU fitting and for step-wise checks) ------------ */
 

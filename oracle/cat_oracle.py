@@ -204,3 +204,24 @@ def affine_with_labels(Yq, labels, gamma, beta, alpha=1.0):
                                       _p(gamma, ctypes.c_float), _p(beta, ctypes.c_float),
                                       float(alpha), _p(out, ctypes.c_float))
     return out
+
+
+def to_bf16(x):
+    """Round fp32 values to bfloat16 (8 significant bits, round to nearest, ties to even) and return
+    them as fp32.  Written out on the bit pattern: add half of the dropped 16 bits' range (plus the
+    parity of the kept part for ties), then clear the low 16 bits.  NaN and infinities pass through."""
+    a = np.ascontiguousarray(x, dtype=np.float32)
+    u = a.view(np.uint32).astype(np.uint64)
+    keep_odd = (u >> 16) & 1
+    r = ((u + 0x7FFF + keep_odd) >> 16) << 16
+    out = (r & 0xFFFFFFFF).astype(np.uint32).view(np.float32).reshape(a.shape)
+    special = ~np.isfinite(a)
+    return np.where(special, a, out)
+
+
+def apply_bf16(Yq, C, gamma, beta):
+    """CAT inference with a bfloat16 result: the fp32 corrected outputs of `apply` (one rounding of
+    gamma*q + beta), rounded once more to bfloat16.  Returns (out as fp32 holding bf16 values, labels,
+    best, second)."""
+    out, labels, best, second = apply(Yq, C, gamma, beta)
+    return to_bf16(out), labels, best, second

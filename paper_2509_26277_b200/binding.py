@@ -34,7 +34,7 @@ class _FastScores(ctypes.Structure):       # cat_fast_scores_t
 
 EXPORTS = [
     "cat_fit_workspace_bytes", "cat_fit", "cat_fit_from", "cat_apply_workspace_bytes",
-    "cat_apply", "cat_apply_blend", "cat_assign", "cat_assign_scores", "cat_assign_noalloc", "cat_cluster_sums",
+    "cat_apply", "cat_apply_blend", "cat_apply_bf16", "cat_assign", "cat_assign_scores", "cat_assign_noalloc", "cat_cluster_sums",
     "cat_fit_shard_begin", "cat_fit_shard_round", "cat_fit_shard_update",
     "cat_pca_workspace_bytes", "cat_pca_fit", "cat_pca_project", "cat_affine_with_labels",
     "cat_fit_pca_workspace_bytes", "cat_fit_pca", "cat_apply_pca_workspace_bytes", "cat_apply_pca",
@@ -92,6 +92,8 @@ def lib():
     L.cat_apply.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     L.cat_apply_blend.argtypes = [vp, i64, i32, i32, vp, vp, vp, f32, vp, vp, vp, sz, vp]
     L.cat_assign.argtypes = [vp, i64, i32, i32, vp, vp, vp, sz, vp]
+    L.cat_apply_bf16.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.cat_apply_bf16.restype = ctypes.c_int
     L.cat_assign_scores.argtypes = [vp, i64, i32, i32, vp, vp, ctypes.POINTER(_FastScores), i32, vp, sz, vp]
     L.cat_assign_scores.restype = ctypes.c_int
     L.cat_assign_noalloc.argtypes = [vp, i64, i32, i32, vp, vp, vp]
@@ -262,6 +264,23 @@ def cat_apply(Yq, centroids, gamma, beta, out=None, want_labels=False, alpha: fl
     else:
         st = lib().cat_apply_blend(*args, ctypes.c_float(alpha), *tail)
     _check(st, "cat_apply")
+    return (out, labels) if want_labels else out
+
+
+def cat_apply_bf16(Yq, centroids, gamma, beta, out=None, want_labels=False, ws=None):
+    """cat_apply_bf16: the corrected rows as a bf16 tensor."""
+    N, D = Yq.shape
+    K = centroids.shape[0]
+    dev = Yq.device
+    if out is None:
+        out = torch.empty((N, D), dtype=torch.bfloat16, device=dev)
+    labels = torch.empty((N,), dtype=torch.int32, device=dev) if want_labels else None
+    ws = workspace("apply", N, D, K, dev) if ws is None else ws
+    st = lib().cat_apply_bf16(_dev(Yq, torch.float32, None, "Yq"), N, D, K, _dev(centroids, torch.float32, (K, D)),
+                              _dev(gamma, torch.float32, (K, D)), _dev(beta, torch.float32, (K, D)),
+                              _dev(out, torch.bfloat16, (N, D), "out"), _dev(labels, torch.int32),
+                              ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream())
+    _check(st, "cat_apply_bf16")
     return (out, labels) if want_labels else out
 
 

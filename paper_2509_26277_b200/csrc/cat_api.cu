@@ -241,6 +241,41 @@ cat_status_t cat_apply(const float *Yq, int64_t N, int32_t D, int32_t K, const f
                            workspace_bytes, stream);
 }
 
+cat_status_t cat_apply_bf16(const float *Yq, int64_t N, int32_t D, int32_t K, const float *centroids,
+                            const float *gamma, const float *beta, void *Y_out_bf16, int32_t *labels_out,
+                            void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!Yq || !centroids || !gamma || !beta || !Y_out_bf16) return CAT_ERR_NULL;
+    cat_status_t st = check_shape(N, D, K, false);
+    if (st != CAT_OK) return st;
+    if (!aligned16(Yq) || !aligned16(centroids) || !aligned16(gamma) || !aligned16(beta) || !aligned16(Y_out_bf16) ||
+        (labels_out && !aligned16(labels_out)))
+        return CAT_ERR_ALIGN;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < cat_apply_workspace_bytes(N, D, K))
+        return CAT_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    AssignWs w = carve_assign(workspace, N, D, K);
+    int32_t *labels = labels_out ? labels_out : w.labels;
+    if (use_tensor_path(N, D, K) && apply_h64_supported(N, D, K)) {
+        // fused: the 64-row-tile kernel writes bf16 with the fast labels; the exact pass settles the
+        // undecided rows' labels, and those rows are written once more
+        CAT_CUDA(launch_centroid_norms(centroids, D, K, w.cnorm, w.ctl, s, true));
+        CAT_CUDA(launch_absmax(centroids, (size_t)K * D, w.hscale, s));
+        CAT_CUDA(launch_half_scale(w.hscale, s));
+        CAT_CUDA(launch_to_half(centroids, (size_t)K * D, w.hscale, w.ch, s));
+        CAT_CUDA(launch_apply_h64(Yq, N, D, K, w.ch, w.hscale, w.cnorm, labels, w.refine_rows, w.cand_rows, w.cand_list, w.ctl,
+                                  gamma, beta, reinterpret_cast<float *>(Y_out_bf16), s, true));
+        CAT_CUDA(launch_refine_both(Yq, N, D, K, centroids, labels, w.cand_rows, w.cand_list, w.refine_rows, w.ctl, nullptr,
+                                    nullptr, nullptr, s));
+        CAT_CUDA(launch_affine_bf16(Yq, N, D, K, labels, gamma, beta, Y_out_bf16, w.refine_rows, w.cand_rows, w.ctl, s));
+        return CAT_OK;
+    }
+    st = run_assign(Yq, N, D, K, centroids, labels, w, nullptr, nullptr, nullptr, s);
+    if (st != CAT_OK) return st;
+    CAT_CUDA(launch_affine_bf16(Yq, N, D, K, labels, gamma, beta, Y_out_bf16, nullptr, nullptr, nullptr, s));
+    return CAT_OK;
+}
+
 cat_status_t cat_assign(const float *Yq, int64_t N, int32_t D, int32_t K, const float *centroids,
                         int32_t *labels_out, void *workspace, size_t workspace_bytes, void *stream)
 {

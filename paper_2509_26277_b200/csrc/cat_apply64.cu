@@ -34,6 +34,8 @@
 // leave.  No TMA multicast; all tensor maps cover this GPU's memory.
 #include "cat_tc.cuh"
 
+#include <cuda_bf16.h>
+
 namespace cat {
 
 namespace {
@@ -132,6 +134,8 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     }
 }
 // One warp streams one row: out = gamma_l * y + beta_l, all loads of a 1024-column step in flight together.
+// OUT_BF16: the corrected row is stored as bf16 (round to nearest even of the fp32 result), 8 bytes per lane and step.
+template <bool OUT_BF16>
 __device__ __forceinline__ void stream_row_plain(const TcParams &p, int64_t row, int l, int lane)
 {
     const int D4 = p.D >> 2;
@@ -139,6 +143,7 @@ __device__ __forceinline__ void stream_row_plain(const TcParams &p, int64_t row,
     const float4 *g4 = reinterpret_cast<const float4 *>(p.gamma) + (size_t)l * D4 + lane;
     const float4 *b4 = reinterpret_cast<const float4 *>(p.beta) + (size_t)l * D4 + lane;
     float4 *o4 = reinterpret_cast<float4 *>(p.out) + (size_t)row * D4 + lane;
+    uint2 *o2 = reinterpret_cast<uint2 *>(p.out) + (size_t)row * D4 + lane;   // bf16 output: four values in 8 bytes
 #pragma unroll 1
     for (int h = 0; h < D4; h += 256) {
         float4 y[8], g[8], bb[8];
@@ -160,7 +165,15 @@ __device__ __forceinline__ void stream_row_plain(const TcParams &p, int64_t row,
                 v.y = fmaf(g[q].y, y[q].y, bb[q].y);
                 v.z = fmaf(g[q].z, y[q].z, bb[q].z);
                 v.w = fmaf(g[q].w, y[q].w, bb[q].w);
-                __stcs(o4 + c, v);
+                if (OUT_BF16) {
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+                    uint2 w;
+                    w.x = *reinterpret_cast<const unsigned int *>(&lo);
+                    w.y = *reinterpret_cast<const unsigned int *>(&hi);
+                    __stcs(o2 + c, w);
+                } else {
+                    __stcs(o4 + c, v);
+                }
             }
         }
     }
@@ -179,6 +192,7 @@ struct H64Params {
     int nh;           // fp16 slabs (64 columns) per row
 };
 
+template <bool OUT_BF16>
 __global__ void __launch_bounds__(H_THREADS, 1)
 apply_h64_kernel(const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapC, H64Params hp)
 {
@@ -516,7 +530,7 @@ apply_h64_kernel(const __grid_constant__ CUtensorMap mapY, const __grid_constant
                 const int64_t nrow = (r + H_STREAM_WARPS < H_ROWS) ? row + H_STREAM_WARPS
                                      : ((unit + unit_step < num_units) ? ((unit + unit_step) * 2 + rank) * H_ROWS + ew : p.N);
                 if (nrow < p.N) prefetch_row_l2(p, nrow, lane);
-                if (row < p.N) stream_row_plain(p, row, sh.lab[b][r], lane);
+                if (row < p.N) stream_row_plain<OUT_BF16>(p, row, sh.lab[b][r], lane);
                 __syncwarp();
                 if (lane == 0) atomicAdd(&sh.rows_streamed, 1);
             }
@@ -573,7 +587,7 @@ cudaError_t launch_absmax(const float *src, size_t n, float *scale, cudaStream_t
 cudaError_t launch_apply_h64(const float *Y, int64_t N, int D, int K, const void *Ch, const float *scale,
                              const float *cnorm, int32_t *labels, int32_t *refine_rows, int32_t *cand_rows,
                              uint64_t *cand_list, Control *ctl, const float *gamma, const float *beta, float *out,
-                             cudaStream_t s)
+                             cudaStream_t s, bool out_bf16)
 {
     H64Params hp{};
     TcParams &p = hp.t;
@@ -624,7 +638,7 @@ cudaError_t launch_apply_h64(const float *Y, int64_t N, int D, int K, const void
     cfg.attrs = attr;
     cfg.numAttrs = 2;
 
-    auto kern = apply_h64_kernel;
+    auto kern = out_bf16 ? apply_h64_kernel<true> : apply_h64_kernel<false>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, carveout)) != cudaSuccess) return e;

@@ -155,7 +155,12 @@ cudaError_t launch_half_scale(float *scale, cudaStream_t s);                    
 cudaError_t launch_apply_h64(const float *Y, int64_t N, int D, int K, const void *Ch, const float *scale,
                              const float *cnorm, int32_t *labels, int32_t *refine_rows, int32_t *cand_rows,
                              uint64_t *cand_list, Control *ctl, const float *gamma, const float *beta, float *out,
-                             cudaStream_t s);
+                             cudaStream_t s, bool out_bf16 = false);   // out_bf16: `out` is a [N, D] bf16 matrix
+// out_bf16[row] = bf16(gamma_l * y + beta_l), l = labels[row]: for all rows (rows == nullptr, n_rows = N) or
+// for the listed rows (two lists, lengths read from ctl: the exact-pass queues).
+cudaError_t launch_affine_bf16(const float *Y, int64_t N, int D, int K, const int32_t *labels, const float *gamma,
+                               const float *beta, void *out_bf16, const int32_t *refine_rows, const int32_t *cand_rows,
+                               const Control *ctl, cudaStream_t s);
 cudaError_t launch_row_norms(const float *Y, int64_t N, int D, float *out, cudaStream_t s);
 // With Yh / Ch / scale (labels only): the fp16 copies of the rows and centroids are the MMA operands.
 cudaError_t launch_assign_tc(const float *Y, int64_t N, int D, int K, const float *C, const float *cnorm,

@@ -16,6 +16,7 @@
 // Everything is deterministic: no floating-point atomics, fixed summation orders.
 #include "cat_internal.cuh"
 
+#include <cuda_bf16.h>
 #include <math_constants.h>
 
 namespace cat {
@@ -374,6 +375,55 @@ __global__ void __launch_bounds__(256) affine_labels_kernel(const float *__restr
     }
 }
 
+// The same with a bf16 result (round to nearest even of the fp32 fused multiply-add), for all rows or
+// for the rows of the two exact-pass queues (whose lengths are read from ctl).
+__global__ void __launch_bounds__(256) affine_bf16_kernel(const float *__restrict__ Y, int64_t N, int D, int K,
+                                                          const int32_t *__restrict__ labels,
+                                                          const float *__restrict__ gamma, const float *__restrict__ beta,
+                                                          __nv_bfloat16 *__restrict__ out,
+                                                          const int32_t *__restrict__ refine_rows,
+                                                          const int32_t *__restrict__ cand_rows, const Control *ctl)
+{
+    const int lane = threadIdx.x & 31;
+    const bool listed = ctl != nullptr;
+    int64_t nref = 0, total = N;
+    if (listed) {
+        nref = ctl->refine_count < N ? ctl->refine_count : N;
+        const int64_t nc = ctl->cand_count < N ? ctl->cand_count : N;
+        total = nref + nc;
+    }
+    const bool vec4 = (D & 3) == 0;
+    for (int64_t q = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); q < total; q += (int64_t)gridDim.x * 8) {
+        const int64_t row = listed ? (int64_t)(q < nref ? refine_rows[q] : cand_rows[q - nref]) : q;
+        if (row < 0 || row >= N) continue;
+        const int l = labels[row];
+        const bool ok = l >= 0 && l < K;
+        const float *y = Y + (size_t)row * D;
+        const float *g = gamma + (size_t)(ok ? l : 0) * D;
+        const float *b = beta + (size_t)(ok ? l : 0) * D;
+        __nv_bfloat16 *o = out + (size_t)row * D;
+        if (vec4) {
+            for (int j = lane; j < (D >> 2); j += 32) {
+                const float4 yv = __ldcs(reinterpret_cast<const float4 *>(y) + j);
+                float4 v = yv;
+                if (ok) {
+                    const float4 gv = __ldg(reinterpret_cast<const float4 *>(g) + j);
+                    const float4 bv = __ldg(reinterpret_cast<const float4 *>(b) + j);
+                    v = make_float4(fmaf(gv.x, yv.x, bv.x), fmaf(gv.y, yv.y, bv.y), fmaf(gv.z, yv.z, bv.z),
+                                    fmaf(gv.w, yv.w, bv.w));
+                }
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+                uint2 w2;
+                w2.x = *reinterpret_cast<const unsigned int *>(&lo);
+                w2.y = *reinterpret_cast<const unsigned int *>(&hi);
+                reinterpret_cast<uint2 *>(o)[j] = w2;
+            }
+        } else {
+            for (int j = lane; j < D; j += 32) o[j] = __float2bfloat16_rn(ok ? fmaf(g[j], y[j], b[j]) : y[j]);
+        }
+    }
+}
+
 int cov_splits(int D)
 {
     const int T = (D + PT - 1) / PT;
@@ -420,6 +470,19 @@ PcaWs carve_pca(void *base, int D)
 inline bool al16(const void *q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
 
 }  // namespace
+
+cudaError_t launch_affine_bf16(const float *Y, int64_t N, int D, int K, const int32_t *labels, const float *gamma,
+                               const float *beta, void *out_bf16, const int32_t *refine_rows, const int32_t *cand_rows,
+                               const Control *ctl, cudaStream_t s)
+{
+    int64_t blocks = (N + 7) / 8;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    affine_bf16_kernel<<<(unsigned)blocks, 256, 0, s>>>(Y, N, D, K, labels, gamma, beta,
+                                                        reinterpret_cast<__nv_bfloat16 *>(out_bf16), refine_rows, cand_rows, ctl);
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace cat
 
 using namespace cat;

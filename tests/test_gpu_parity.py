@@ -464,6 +464,26 @@ def test_alpha_blend(alpha):
         assert torch.equal(out, B.cat_apply(dev(Yq), dev(C), dev(g), dev(b)))
 
 
+@pytest.mark.parametrize("n,d,k", [(3000, 1024, 64), (1111, 1000, 16), (500, 36, 5), (5000, 256, 200), (70, 130, 3)])
+def test_apply_with_bf16_output(n, d, k):
+    """cat_apply_bf16 on shapes that take the fused 64-row-tile kernel and on shapes that take the
+    assignment followed by a second pass: labels as cat_apply, outputs equal to the oracle's bit for bit."""
+    rng = np.random.default_rng(n + d + k)
+    cen = (rng.normal(size=(k, d)) * 2).astype(np.float32)
+    Yq = (cen[rng.integers(0, k, size=n)] + rng.normal(size=(n, d))).astype(np.float32)
+    Yq[: n // 4] = (0.5 * (cen[rng.integers(0, k, size=n // 4)] + cen[rng.integers(0, k, size=n // 4)])
+                    + 1e-4 * rng.normal(size=(n // 4, d))).astype(np.float32)     # undecided rows: midway between centroids
+    G = rng.normal(size=(k, d)).astype(np.float32)
+    Bt = rng.normal(size=(k, d)).astype(np.float32)
+    want, lab, best, second = O.apply_bf16(Yq, cen, G, Bt)
+    out, glab = B.cat_apply_bf16(dev(Yq), dev(cen), dev(G), dev(Bt), want_labels=True)
+    assert out.dtype == torch.bfloat16
+    _, n_diff = labels_match(host(glab), lab, best, second, "labels (bf16 output)")
+    if n_diff:
+        want = O.to_bf16(O.affine_with_labels(Yq, host(glab), G, Bt))
+    np.testing.assert_array_equal(out.float().cpu().numpy(), want)
+
+
 def test_step_level_moments_and_solve():
     Yq, Yfp = _rand(13, 3000, 48), _rand(14, 3000, 48)
     labels = np.random.default_rng(15).integers(0, 10, size=3000).astype(np.int32)

@@ -438,3 +438,18 @@ def test_fit_rejects_bad_shapes():
         O.fit(Y, Y, 4, 1)
     with pytest.raises(ValueError):
         O.fit(Y, Y, 0, 1)
+
+
+def test_bf16_rounding_ties_to_even_and_matches_torch():
+    import torch
+    # 1 + 2^-8 lies halfway between 1 and 1 + 2^-7: the tie goes to the even mantissa (1); 1 + 3 * 2^-8 goes up
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, 1.0 + 3 * 2.0 ** -8, -1.0 - 2.0 ** -8, 0.0,
+                  3.0e38, 1e-40, np.inf], np.float32)
+    want = np.array([1.0, 1.0, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -6, -1.0, 0.0, 3.0e38, 1e-40, np.inf], np.float32)
+    got = O.to_bf16(x)
+    assert got[0] == 1.0 and got[1] == 1.0 and got[2] == np.float32(1.0 + 2.0 ** -7)
+    assert got[3] == np.float32(1.0 + 2.0 ** -6) and got[4] == -1.0 and got[5] == 0.0 and np.isinf(got[8])
+    r = np.random.default_rng(0).normal(size=100000).astype(np.float32) * np.float32(1e3)
+    ref = torch.from_numpy(r).to(torch.bfloat16).to(torch.float32).numpy()
+    np.testing.assert_array_equal(O.to_bf16(r), ref)
+    assert (np.abs(O.to_bf16(r) - r) <= np.abs(r) * 2.0 ** -8).all()      # within half a bf16 ulp

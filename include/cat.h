@@ -397,6 +397,18 @@ cat_status_t cat_selftest_wait_timeout(void *workspace, size_t workspace_bytes, 
 void cat_set_tensor_core_min_k(int32_t min_k);
 int32_t cat_get_tensor_core_min_k(void);
 
+/* Small problems (D one of 32, 64, 128; K <= 128, and K * D <= 4096 for fitting; at least 128
+ * rows; K >= the tensor-core threshold above) have persistent single-launch kernels: scores on the
+ * tensor cores, undecided rows settled in fp64 inside the kernel, and for fitting the per-cluster
+ * sums kept on chip and combined across the grid in a fixed order, all rounds in one launch.
+ * mask bit 0: the whole of cat_apply (Algorithm 2) runs that way (default: on -- it is the faster
+ * form where it applies).  mask bit 1: so do the K-Means rounds of cat_fit / cat_fit_from
+ * (Algorithm 1, step 2; calls without per-round diagnostics) (default: off -- measured slower than
+ * the general multi-launch path; kept as a tested alternative).  Same labels either way; sums that
+ * agree to fp64 rounding.  A PROCESS-WIDE tuning and test hook like the one above. */
+void cat_set_small_problem_kernels(int32_t mask);
+int32_t cat_get_small_problem_kernels(void);
+
 /* 1 if the tensor-core kernels can run in this process (the driver hands out the tensor-map
  * encoder they need), 0 if not.  When it is 0 every call takes the fp32-pipe kernels, which
  * give the same results about ten times slower for large K; callers that depend on the speed

@@ -43,6 +43,7 @@ EXPORTS = [
     "cat_apply_host", "cat_fit_host_workspace_bytes", "cat_fit_host", "cat_workspace_report",
     "cat_selftest_wait_timeout",
     "cat_set_tensor_core_min_k", "cat_get_tensor_core_min_k", "cat_tensor_path_available",
+    "cat_set_small_problem_kernels", "cat_get_small_problem_kernels",
     "cat_set_apply_column_split", "cat_get_apply_column_split", "cat_status_string",
     "cat_last_cuda_error", "cat_version", "cat_kernel_launches",
 ]
@@ -133,6 +134,9 @@ def lib():
     L.cat_set_tensor_core_min_k.argtypes = [i32]
     L.cat_set_tensor_core_min_k.restype = None
     L.cat_get_tensor_core_min_k.restype = i32
+    L.cat_set_small_problem_kernels.argtypes = [i32]
+    L.cat_set_small_problem_kernels.restype = None
+    L.cat_get_small_problem_kernels.restype = i32
     L.cat_tensor_path_available.restype = i32
     L.cat_set_apply_column_split.argtypes = [i32]
     L.cat_set_apply_column_split.restype = None
@@ -552,6 +556,16 @@ def cat_set_tensor_core_min_k(min_k: int) -> None:
 
 def cat_get_tensor_core_min_k() -> int:
     return int(lib().cat_get_tensor_core_min_k())
+
+
+def cat_set_small_problem_kernels(mask: int) -> None:
+    """Process-wide switch of the persistent single-launch kernels for small shapes:
+    bit 0 = inference (default on), bit 1 = the K-Means rounds of a fit (default off)."""
+    lib().cat_set_small_problem_kernels(int(mask))
+
+
+def cat_get_small_problem_kernels() -> int:
+    return int(lib().cat_get_small_problem_kernels())
 
 
 def cat_tensor_path_available() -> bool:

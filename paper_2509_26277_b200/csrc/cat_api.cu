@@ -80,6 +80,11 @@ FitWs carve_fit(void *base, int64_t N, int D, int K)
     w.meanQ = c.take<double>(KD);
     w.meanF = c.take<double>(KD);
     w.counts = c.take<int64_t>((size_t)K);
+    if (small_fit_supported(N, D, K)) {
+        // per-CTA partial sums and sizes of the persistent small-problem kernel
+        w.small_part = c.take<double>(small_part_doubles(D, K));
+        w.small_counts = c.take<int32_t>(small_part_counts(K));
+    }
     w.bytes = align_up(c.off, 256);
     return w;
 }
@@ -99,10 +104,21 @@ static cat_status_t check_shape(int64_t N, int32_t D, int32_t K, bool need_n_ge_
     } while (0)
 
 static std::atomic<int> g_tc_min_k{32};
+static std::atomic<int> g_small_kernels{1};   // bit 0: inference, bit 1: the K-Means rounds of a fit
 
 static bool use_tensor_path(int64_t N, int D, int K)
 {
     return K >= g_tc_min_k.load(std::memory_order_relaxed) && tc_supported(N, D, K);
+}
+
+// the persistent single-launch kernels take the small shapes they support, unless switched off
+static bool use_small_fit(int64_t N, int D, int K)
+{
+    return (g_small_kernels.load(std::memory_order_relaxed) & 2) && use_tensor_path(N, D, K) && small_fit_supported(N, D, K);
+}
+static bool use_small_apply(int64_t N, int D, int K)
+{
+    return (g_small_kernels.load(std::memory_order_relaxed) & 1) && use_tensor_path(N, D, K) && small_apply_supported(N, D, K);
 }
 
 // norms -> fast assignment (tensor cores for large K, fp32 pipes otherwise) -> exact pass for
@@ -114,6 +130,12 @@ static cat_status_t run_assign(const float *Y, int64_t N, int D, int K, const fl
                                const void *Yh = nullptr, void *Ch = nullptr, const float *hscale = nullptr,
                                bool centroids_ready = false, const FastOut *fast = nullptr)
 {
+    if (out && labels && top_level && !fast && use_small_apply(N, D, K)) {
+        // small problems: everything in one persistent launch (exact decisions included)
+        CAT_CUDA(launch_reset_control(w.ctl, s));
+        CAT_CUDA(launch_small_apply(Y, N, D, K, C, gamma, beta, out, labels, w.ctl, s));
+        return CAT_OK;
+    }
     // centroids_ready: the centroid update that produced C has already left its norms, its fp16
     // copy and empty exact-pass queues in the workspace
     if (!centroids_ready) CAT_CUDA(launch_centroid_norms(C, D, K, w.cnorm, w.ctl, s, top_level));
@@ -359,6 +381,15 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     CAT_CUDA(cudaMemcpyAsync(C, init_centroids ? init_centroids : Yq, KD * sizeof(float),
                              cudaMemcpyDeviceToDevice, s));
 
+    // Small problems without per-round diagnostics: every round, the final assignment and the
+    // per-cluster sums and sizes that follow its labels come from one persistent launch.
+    const bool small = !diag && use_small_fit(N, D, K);
+    if (small) {
+        unsigned int bar_count = 0;   // (the control block was reset above)
+        CAT_CUDA(launch_small_fit(Yq, N, D, K, C, iters + 1, false, labels, w.small_part, w.small_counts, w.sumQ,
+                                  w.counts, w.a.ctl, &bar_count, s));
+    }
+
     const bool tc = use_tensor_path(N, D, K);
     // Yq is fixed over the fit: its row norms, and where the shape allows an fp16 copy for the
     // tensor cores, are made once
@@ -366,7 +397,8 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     // largest magnitude of Yq, which sets the fp16 scale; caller-provided ones could overflow it)
     const bool half = tc && !init_centroids && tc_half_supported(N, D, K);
     const void *Yh = half ? w.yh : nullptr;
-    if (half) CAT_CUDA(launch_half_shadow(Yq, N, D, w.a.ynorm2, w.hscale, w.yh, s));
+    if (small) {
+    } else if (half) CAT_CUDA(launch_half_shadow(Yq, N, D, w.a.ynorm2, w.hscale, w.yh, s));
     else if (tc) CAT_CUDA(launch_row_norms(Yq, N, D, w.a.ynorm2, s));
 
     // Lloyd rounds.  Two label buffers alternate so that a round sees the previous round's
@@ -374,6 +406,7 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
     // sizes start at zero with "no previous label" (-1) for every row.
     const int diag_recorded = iters + 1 < CAT_DIAG_MAX_ROUNDS ? iters + 1 : CAT_DIAG_MAX_ROUNDS;
     int32_t *lab[2] = {labels, w.labels_prev};
+    if (!small) {
     CAT_CUDA(cudaMemsetAsync(lab[(iters & 1) ^ 1], 0xFF, (size_t)N * sizeof(int32_t), s));
     CAT_CUDA(cudaMemsetAsync(w.sumQ, 0, KD * sizeof(double), s));
     CAT_CUDA(cudaMemsetAsync(w.counts, 0, (size_t)K * sizeof(int64_t), s));
@@ -407,6 +440,7 @@ cat_status_t cat_fit_from(const float *Yq, const float *Yfp, int64_t N, int32_t 
                                      2 * K, gd, w.segpart, s));
         CAT_CUDA(launch_segment_combine(w.segpart, w.seg_start, w.counts, D, K, true, w.sumQ, nullptr, nullptr, s));
     }
+    }   // !small
     CAT_CUDA(launch_means_from_sums(w.sumQ, w.counts, D, K, meanQ, s));
     st = run_sort(labels, N, D, K, w, w.counts, s);
     if (st != CAT_OK) return st;
@@ -605,6 +639,9 @@ void cat_set_tensor_core_min_k(int32_t min_k)
 }
 
 int32_t cat_get_tensor_core_min_k(void) { return g_tc_min_k.load(std::memory_order_relaxed); }
+
+void cat_set_small_problem_kernels(int32_t mask) { g_small_kernels.store(mask & 3, std::memory_order_relaxed); }
+int32_t cat_get_small_problem_kernels(void) { return g_small_kernels.load(std::memory_order_relaxed); }
 
 int32_t cat_tensor_path_available(void) { return tc_supported(1, 4, 1) ? 1 : 0; }
 

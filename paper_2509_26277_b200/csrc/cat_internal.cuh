@@ -70,7 +70,7 @@ struct Control {
     int64_t refined_total;       // running total over assignments
     int64_t refined_last;        // rows of the latest finished assignment that took an exact pass
     int32_t cand_count;          // rows queued with a short candidate list by the current assignment
-    int32_t pad0;
+    uint32_t grid_bar;           // arrival counter of the grid-wide barrier of the persistent small-problem kernel
     int64_t pad[4];
 };
 
@@ -116,6 +116,8 @@ struct FitWs {
     double *sumQ, *sumF, *var, *cov;   // [K*D] each
     double *meanQ, *meanF;             // [K*D] each
     int64_t *counts;       // [K]
+    double *small_part;    // [SMALL_MAX_GRID][K*D] per-CTA sums of the persistent small-problem kernel (or null)
+    int32_t *small_counts; // [SMALL_MAX_GRID][K+1]
     size_t bytes;
 };
 FitWs carve_fit(void *base, int64_t N, int D, int K);
@@ -138,6 +140,19 @@ cudaError_t launch_assign(const float *Y, int64_t N, int D, int K, const float *
 cudaError_t launch_refine(const float *Y, int64_t N, int D, int K, const float *C,
                           int32_t *labels, const int32_t *refine_rows, Control *ctl,
                           const float *gamma, const float *beta, float *out, cudaStream_t s);
+
+// Persistent single-launch kernels for small problems (D in {32, 64, 128}, K <= 128): a run of
+// Lloyd rounds with the per-cluster sums in registers and a grid-wide combine, and inference.
+constexpr int SMALL_MAX_GRID = 160;   // CTAs the partial-sum planes are sized for
+bool small_fit_supported(int64_t N, int D, int K);
+bool small_apply_supported(int64_t N, int D, int K);
+size_t small_part_doubles(int D, int K);
+size_t small_part_counts(int K);
+cudaError_t launch_small_fit(const float *Y, int64_t N, int D, int K, float *C, int passes, bool update_last,
+                             int32_t *labels, double *part, int32_t *part_counts, double *sums, int64_t *counts,
+                             Control *ctl, unsigned int *bar_count, cudaStream_t s);
+cudaError_t launch_small_apply(const float *Y, int64_t N, int D, int K, const float *C, const float *gamma,
+                               const float *beta, float *out, int32_t *labels, Control *ctl, cudaStream_t s);
 
 // Tensor-core (tcgen05, TF32) variant of launch_assign; ynorm2 is needed when out == nullptr.
 bool tc_supported(int64_t N, int D, int K);

@@ -1064,9 +1064,11 @@ __global__ void reset_control_kernel(Control *ctl)
 {
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         ctl->refine_count = 0;
+        ctl->cand_count = 0;
         ctl->device_status = CAT_OK;
         ctl->refined_total = 0;
         ctl->refined_last = 0;
+        ctl->grid_bar = 0;
     }
 }
 

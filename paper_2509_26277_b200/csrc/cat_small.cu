@@ -1,0 +1,796 @@
+// Small problems (rows of at most 128 columns, at most 128 centroids): a whole Lloyd round -- and
+// a whole run of rounds -- of the K-Means step of the fitting algorithm (Algorithm 1, step 2), or
+// the whole of inference (Algorithm 2: nearest centroid, then gamma_l * y + beta_l), in ONE
+// persistent launch of one CTA per SM.
+//
+// At these shapes the bytes are few (a round reads the rows once: tens of MB) and a chain of
+// short kernels spends its time between launches.  Here a CTA walks its own 128-row tiles:
+//
+//   warp 0      TMA producer: a row tile (128 x D fp32, 128-byte swizzle) per ring stage
+//   warp 1      issues the TF32 tcgen05.mma of the tile against all centroids (accumulator in
+//               TMEM, one buffer per ring stage)
+//   warps 4-11  score warps, two sets of four that take alternate tiles: read the scores from
+//               TMEM, keep the four smallest keys per row and take the certainty test; the rows that
+//               fail it are settled at once by the warp together (fp64 direct form over the listed
+//               candidates, or over all K), so the labels that leave these warps are final
+//   warps 12-27 worker warps: either add the tile's rows to per-cluster fp64 sums in shared memory
+//               (warp w owns the clusters k = w mod 16, a lane owns D / 32 columns), or write
+//               gamma_l * y + beta_l.
+//
+// After its last tile a CTA stores its partial sums; a bounded grid-wide barrier later every warp
+// of the grid adds up, in a fixed order, the partials of a few (cluster, column) pairs and writes
+// the new centroid entry.  A second barrier publishes the centroids for the next round.  Every
+// order of summation is fixed by the launch geometry, so results repeat bit for bit.
+//
+// The launch is cooperative (all CTAs resident), and every wait -- on an mbarrier or on the grid
+// barrier -- gives up after a time limit, raises the device status and lets the kernel return.
+//
+// Measured on 200 704 x 64 rows, K = 64: inference 74 us against 85 us for the general path; a
+// Lloyd round 81 us against 57 us (per-tile handoffs between the warp roles, the exact pass on
+// about 15 % of the rows -- TF32 scores -- and two grid barriers a round cost more than the launches
+// they replace), so fitting takes this kernel only on request.
+#include "cat_tc.cuh"
+
+namespace cat {
+namespace {
+
+constexpr int SM_ROWS = 128;                 // rows per tile
+constexpr int SM_MAX_STAGES = 4;
+constexpr unsigned SM_POLL_SLEEP_NS = 100;
+constexpr int SM_FIRST_SCORE_WARP = 4;
+constexpr int SM_FIRST_WORKER_WARP = 12;     // warps 4-11: two sets of four score warps
+constexpr int SM_WORKERS = 16;
+constexpr int SM_WARPS = SM_FIRST_WORKER_WARP + SM_WORKERS;   // 28
+constexpr int SM_THREADS = 32 * SM_WARPS;                     // 896
+
+struct ExactBest {
+    double d;
+    int k;
+};
+
+struct SmallParams {
+    const float *Y;          // [N, D]
+    float *C;                // [K, D] centroids, updated in place by a round
+    int32_t *labels;         // [N] labels of the last pass (written in that pass only; may be null)
+    double *part;            // [grid, K * D] partial sums of a CTA
+    int32_t *part_counts;    // [grid, K + 1] partial sizes of a CTA, then its count of queued rows
+    double *sums;            // [K * D] per-cluster sums of the last pass
+    int64_t *counts;         // [K]
+    const float *gamma;      // inference only
+    const float *beta;
+    float *out;
+    Control *ctl;
+    unsigned int bar_base;   // value of the counter when this launch starts
+    int64_t N;
+    int D;
+    int K;
+    int npad;                // K rounded up to 32
+    int stages;              // ring depth, a power of two
+    int stage_shift;         // its logarithm
+    int tmem_cols;
+    int passes;              // assignments to run
+    int update_last;         // does the last pass move the centroids too?
+};
+
+struct SmallShared {
+    uint64_t a_full[SM_MAX_STAGES];
+    uint64_t a_empty[SM_MAX_STAGES];
+    uint64_t tmem_full[SM_MAX_STAGES];
+    uint64_t lab_full[SM_MAX_STAGES];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int queued_pass;                        // rows this CTA queued in the current pass
+    float cmax2;
+    float cn[128];
+    int32_t label[SM_MAX_STAGES][SM_ROWS];
+};
+
+// byte offset of element (row, col) in a 128-byte-swizzled operand tile of `rows` rows: 32-column
+// slabs one after another, rows 128 B apart inside a slab, 16-byte chunks XORed with the row
+__device__ __forceinline__ uint32_t swz(int rows, int row, int col)
+{
+    return (uint32_t)((col >> 5) * rows * 128 + row * 128 + ((((col & 31) >> 2) ^ (row & 7)) << 4) + ((col & 3) << 2));
+}
+
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int *p)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Grid-wide barrier for a cooperative launch: the whole CTA calls it.  `target` is the counter
+// value once every CTA has arrived.  False after a timeout or when any CTA has given up (the
+// device status is raised then, and every CTA sees it here at the latest).
+__device__ __forceinline__ bool grid_barrier(const SmallParams &p, unsigned int target, volatile int *abort_flag)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&p.ctl->grid_bar, 1u);
+        uint64_t t0 = 0;
+        for (uint32_t it = 0;; ++it) {
+            // (wrap-safe comparison: the counter only grows)
+            if ((int)(ld_acquire_gpu(&p.ctl->grid_bar) - target) >= 0) break;
+            if ((it & 15u) == 15u) {
+                if (*abort_flag || *(volatile int *)&p.ctl->device_status != (int)CAT_OK) { *abort_flag = 1; break; }
+                uint64_t now = global_timer();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > TC_TIMEOUT_NS) {
+                    *abort_flag = 1;
+                    atomicExch(&p.ctl->device_status, (int)CAT_ERR_DEVICE_TIMEOUT);
+                    break;
+                }
+            }
+        }
+        __threadfence();
+    }
+    __syncthreads();
+    return *abort_flag == 0;
+}
+
+// Bounded waits of this kernel.  Some twenty warps of a CTA are waiting at any time; a failed
+// poll is followed by a short pause, which leaves the issue slots to the warps that have work
+// (it costs nothing measurable).  Every lane of a waiting warp polls: a variant in which lane 0
+// polled alone and told the others by a shuffle ran the kernel at half the speed.
+__device__ __forceinline__ bool wait_one(uint32_t bar, uint32_t parity, volatile int *abort_flag, Control *ctl)
+{
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        __nanosleep(SM_POLL_SLEEP_NS);
+        if ((it & 63u) == 63u) {
+            const uint64_t now = global_timer();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > TC_TIMEOUT_NS) {
+                *abort_flag = 1;
+                atomicExch(&ctl->device_status, (int)CAT_ERR_DEVICE_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+// every lane polls; the warp goes on only if all lanes succeeded
+__device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, Control *ctl, int lane)
+{
+    (void)lane;
+    return __all_sync(0xffffffffu, wait_one(bar, parity, abort_flag, ctl));
+}
+
+// CPL consecutive columns of one row of a swizzled tile (CPL = 1, 2 or 4: inside one 16-byte chunk)
+template <int CPL>
+__device__ __forceinline__ void load_cols(const unsigned char *tile, int rows, int row, int col0, float (&v)[CPL])
+{
+    const unsigned char *src = tile + swz(rows, row, col0);
+    if (CPL == 4) {
+        const float4 t = *reinterpret_cast<const float4 *>(src);
+        v[0] = t.x; v[1] = t.y; v[2 % CPL] = t.z; v[3 % CPL] = t.w;
+    } else if (CPL == 2) {
+        const float2 t = *reinterpret_cast<const float2 *>(src);
+        v[0] = t.x; v[1 % CPL] = t.y;
+    } else {
+        v[0] = *reinterpret_cast<const float *>(src);
+    }
+}
+
+__device__ __forceinline__ double warp_sum_f64(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Exact choice among up to four centroids for one row, by one warp: lanes 8g .. 8g + 7 form
+// ||y - c||^2 in fp64 (direct form) for candidate g -- a lane takes D / 8 consecutive columns in
+// order, then a fixed three-step tree inside the group -- and the four groups are compared:
+// the smallest distance wins, the lowest index among equals.  A candidate index >= K is unused
+// (distance +inf).  The result is the same in every lane.
+template <int CPL>
+__device__ __forceinline__ ExactBest best_of_four(const unsigned char *atile, const unsigned char *btile, int npad,
+                                                  int K, int r, int k_mine, int lane)
+{
+    const int sub = lane & 7;
+    const bool valid = k_mine < K;
+    const int kc = valid ? k_mine : 0;
+    double s = 0.0;
+#pragma unroll
+    for (int i = 0; i < CPL; ++i) {
+        const int col = 4 * (sub * CPL + i);
+        const float4 y = *reinterpret_cast<const float4 *>(atile + swz(SM_ROWS, r, col));
+        const float4 c = *reinterpret_cast<const float4 *>(btile + swz(npad, kc, col));
+        double d;
+        d = (double)y.x - (double)c.x; s = fma(d, d, s);
+        d = (double)y.y - (double)c.y; s = fma(d, d, s);
+        d = (double)y.z - (double)c.z; s = fma(d, d, s);
+        d = (double)y.w - (double)c.w; s = fma(d, d, s);
+    }
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    ExactBest b;
+    b.d = valid ? s : CUDART_INF;
+    b.k = valid ? k_mine : 0x7FFFFFFF;
+#pragma unroll
+    for (int o = 8; o < 32; o <<= 1) {
+        const double d2 = __shfl_xor_sync(0xffffffffu, b.d, o);
+        const int k2 = __shfl_xor_sync(0xffffffffu, b.k, o);
+        if (d2 < b.d || (d2 == b.d && k2 < b.k) || (b.d != b.d && d2 == d2)) { b.d = d2; b.k = k2; }
+    }
+    return b;
+}
+
+// APPLY: inference (one pass, no sums, no grid barrier).  CPL = D / 32 columns per lane,
+
+template <bool APPLY, int CPL>
+__global__ void __launch_bounds__(SM_THREADS, 1)
+small_kernel(const __grid_constant__ CUtensorMap mapA, SmallParams p)
+{
+    pdl_enter();
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles_base = (raw + 1023u) & ~1023u;   // the 128-byte swizzle wants 1024-byte alignment
+    unsigned char *tiles = smem_raw + (tiles_base - raw);
+    const int a_bytes = SM_ROWS * p.D * 4;                // one row tile: D / 32 slabs of 16 KB
+    const int b_bytes = p.npad * p.D * 4;
+    const int na = p.stages;
+    unsigned char *btile = tiles + (size_t)na * a_bytes;
+    const uint32_t b_base = tiles_base + (uint32_t)(na * a_bytes);
+    // per-cluster sums (fp64) and sizes of this CTA's rows in the current pass (fitting only)
+    double *sacc = reinterpret_cast<double *>(btile + b_bytes);
+    int *scnt = reinterpret_cast<int *>(sacc + (APPLY ? 0 : p.K * p.D));
+    SmallShared &sh = *reinterpret_cast<SmallShared *>(scnt + (APPLY ? 0 : 128));
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int *abort_flag = &sh.abort_flag;
+    const int num_tiles = (int)((p.N + SM_ROWS - 1) / SM_ROWS);
+    const int nslabs = p.D >> 5;
+    const int G = (int)gridDim.x;
+
+    if (tid == 0) {
+        for (int s = 0; s < na; ++s) {
+            mbar_init(smem_u32(&sh.a_full[s]), 1);
+            mbar_init(smem_u32(&sh.a_empty[s]), SM_WORKERS);
+            mbar_init(smem_u32(&sh.tmem_full[s]), 1);
+            mbar_init(smem_u32(&sh.lab_full[s]), 4);
+        }
+        mbar_init(smem_u32(&sh.drain), 1);
+        sh.abort_flag = 0;
+        sh.queued_pass = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (!APPLY) {
+        for (int i = tid; i < p.K * p.D; i += SM_THREADS) sacc[i] = 0.0;
+        if (tid < 128) scnt[tid] = 0;
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh.tmem_base), (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    // tiles this CTA has been through, all passes: ring stage = count mod depth, phase = next bit
+    uint32_t tcount = 0;
+    unsigned int bar_next = p.bar_base;
+    bool alive = true;
+
+    for (int pass = 0; pass < p.passes && alive; ++pass) {
+        // ---------------------------------------------------------------- centroids of this pass
+        // into the swizzled operand tile (rows beyond K are zero), read past L1: other CTAs wrote them
+        for (int i = tid; i < p.npad * (p.D >> 2); i += SM_THREADS) {
+            const int k = i / (p.D >> 2), c4 = i - k * (p.D >> 2);
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (k < p.K) v = __ldcg(reinterpret_cast<const float4 *>(p.C) + (size_t)k * (p.D >> 2) + c4);
+            *reinterpret_cast<float4 *>(btile + swz(p.npad, k, c4 * 4)) = v;
+        }
+        __syncthreads();
+        // squared norms in fp64, rounded up; beyond K a huge finite value
+        for (int k = warp; k < 128; k += SM_WARPS) {
+            float cn = TC_KEY_INIT;
+            if (k < p.K) {
+                float c[CPL];
+                load_cols<CPL>(btile, p.npad, k, lane * CPL, c);
+                double s = 0.0;
+#pragma unroll
+                for (int j = 0; j < CPL; ++j) s = fma((double)c[j], (double)c[j], s);
+                cn = __double2float_ru(warp_sum_f64(s));
+            }
+            if (lane == 0) sh.cn[k] = cn;
+        }
+        // the MMA reads the tile through the async proxy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            float m = 0.f;
+            for (int k = 0; k < p.K; ++k) m = fmaxf(m, sh.cn[k]);
+            sh.cmax2 = m;
+        }
+        __syncthreads();
+        const float cmax2 = sh.cmax2;
+
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer
+            if (lane == 0) {
+                for (int tile = (int)blockIdx.x; tile < num_tiles; tile += G, ++tcount) {
+                    const int rs = (int)(tcount & (uint32_t)(na - 1));
+                    const uint32_t rph = (tcount >> p.stage_shift) & 1u;
+                    if (!wait_one(smem_u32(&sh.a_empty[rs]), rph ^ 1u, abort_flag, p.ctl)) break;
+                    const uint32_t full = smem_u32(&sh.a_full[rs]);
+                    mbar_arrive_expect_tx(full, (uint32_t)a_bytes);
+                    for (int sl = 0; sl < nslabs; ++sl)
+                        tma_load_2d(tiles_base + (uint32_t)(rs * a_bytes + sl * TC_A_BYTES), &mapA, full, sl * 32,
+                                    (int)(tile * SM_ROWS));
+                }
+            }
+        } else if (warp == 1) {
+            // ------------------------------------------------------------ MMA issuer
+            if (lane == 0) {
+                const uint32_t idesc = make_idesc(SM_ROWS, p.npad, 2u);
+                for (int tile = (int)blockIdx.x; tile < num_tiles; tile += G, ++tcount) {
+                    const int rs = (int)(tcount & (uint32_t)(na - 1));
+                    const uint32_t rph = (tcount >> p.stage_shift) & 1u;
+                    // (the accumulator of this stage is free: the stage itself was released by the
+                    // workers, who run after the score warps, before the producer refilled it)
+                    if (!wait_one(smem_u32(&sh.a_full[rs]), rph, abort_flag, p.ctl)) break;
+                    tc_fence_after();
+                    const uint32_t accum_at = tmem_base + (uint32_t)(rs * p.npad);
+                    for (int sl = 0; sl < nslabs; ++sl) {
+                        const uint64_t adesc = make_smem_desc(tiles_base + (uint32_t)(rs * a_bytes + sl * TC_A_BYTES));
+                        const uint64_t bdesc = make_smem_desc(b_base + (uint32_t)(sl * p.npad * 128));
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)   // 8 tf32 = 32 B per MMA: +2 in 16-byte units
+                            mma_tf32(accum_at, adesc + 2 * kk, bdesc + 2 * kk, idesc, (sl > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&sh.tmem_full[rs]));
+                }
+            }
+        } else if (warp >= SM_FIRST_SCORE_WARP && warp < SM_FIRST_WORKER_WARP) {
+            // ------------------------------------------------------------ score warps
+            // Two sets of four warps take alternate tiles.  A thread owns one row: its norm, its four
+            // smallest keys, the certainty test.  Rows that fail the test are then settled exactly by
+            // the warp together, one row at a time, so the labels that leave here are final.
+            const int set = (warp - SM_FIRST_SCORE_WARP) >> 2;
+            const int quarter = warp & 3;   // the TMEM lanes this warp may read
+            const int r = quarter * 32 + lane;
+            int settled = 0;
+            for (int tile = (int)blockIdx.x; tile < num_tiles; tile += G, ++tcount) {
+                if ((int)(tcount & 1u) != set) continue;
+                const int rs = (int)(tcount & (uint32_t)(na - 1));
+                const uint32_t rph = (tcount >> p.stage_shift) & 1u;
+                const int64_t row = (int64_t)tile * SM_ROWS + r;
+                const unsigned char *atile = tiles + (size_t)rs * a_bytes;
+                // (the tile itself was written through the async proxy: its own barrier makes it visible)
+                if (!wait_warp(smem_u32(&sh.a_full[rs]), rph, abort_flag, p.ctl, lane)) break;
+                // squared norm of this thread's row, for the error bound (fp32; over-estimated below)
+                float yn2;
+                {
+                    // (four partial sums: one chain of D dependent FMAs would cost more than the key scan)
+                    float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+                    for (int c4 = 0; c4 < 8 * CPL; ++c4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(atile + swz(SM_ROWS, r, c4 * 4));
+                        q0 = fmaf(v.x, v.x, q0);
+                        q1 = fmaf(v.y, v.y, q1);
+                        q2 = fmaf(v.z, v.z, q2);
+                        q3 = fmaf(v.w, v.w, q3);
+                    }
+                    yn2 = (q0 + q1) + (q2 + q3);
+                }
+                if (!wait_warp(smem_u32(&sh.tmem_full[rs]), rph, abort_flag, p.ctl, lane)) break;
+                tc_fence_after();
+                float b1 = TC_KEY_INIT, b2 = TC_KEY_INIT, b3 = TC_KEY_INIT, b4 = TC_KEY_INIT;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(rs * p.npad);
+                uint32_t ra[16], rb[16];
+                tmem_ld16_issue(taddr, ra);
+                for (int c = 0; c < p.npad; c += 32) {
+                    tmem_ld_wait16(ra);
+                    tmem_ld16_issue(taddr + (uint32_t)(c + 16), rb);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        key_insert(make_key(fmaf(-2.f, __uint_as_float(ra[j]), sh.cn[c + j]), c + j), b1, b2, b3, b4);
+                    tmem_ld_wait16(rb);
+                    if (c + 32 < p.npad) tmem_ld16_issue(taddr + (uint32_t)(c + 32), ra);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        key_insert(make_key(fmaf(-2.f, __uint_as_float(rb[j]), sh.cn[c + 16 + j]), c + 16 + j), b1, b2, b3, b4);
+                }
+                int lab = -1;
+                // Candidates of an undecided row, one bit per centroid: those whose key lies within the
+                // limit of the best.  When the fourth smallest key is still inside the limit the row's
+                // scores are read once more from TMEM to find them all.
+                uint32_t mk[4] = {0u, 0u, 0u, 0u};
+                bool undecided = false, wide = false;
+                float lim = 0.f;
+                if (row < p.N) {
+                    lab = key_label(b1, p.K);
+                    lim = 2.f * tc_error_bound(p.D, yn2 * 1.0001f, cmax2);
+                    if (p.K > 1 && !((b2 - b1) > lim)) {
+                        undecided = true;
+                        wide = !((b4 - b1) > lim) && p.K > 4;
+                        if (!wide) {
+                            const float bk[4] = {b1, b2, b3, b4};
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                const int k = key_index(bk[t]);
+                                if (t < p.K && !((bk[t] - b1) > lim)) {
+#pragma unroll
+                                    for (int q = 0; q < 4; ++q)
+                                        if ((k >> 5) == q) mk[q] |= 1u << (k & 31);
+                                }
+                            }
+                        }
+                    }
+                }
+                if (__any_sync(0xffffffffu, wide)) {
+                    // (the TMEM loads are warp-wide; only the rows that asked use what they return)
+#pragma unroll
+                    for (int c = 0; c < 128; c += 16) {
+                        if (c < p.npad) {
+                            tmem_ld16_issue(taddr + (uint32_t)c, ra);
+                            tmem_ld_wait16(ra);
+                            uint32_t bits = 0;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float key = make_key(fmaf(-2.f, __uint_as_float(ra[j]), sh.cn[c + j]), c + j);
+                                if (c + j < p.K && !((key - b1) > lim)) bits |= 1u << j;
+                            }
+                            if (wide) mk[c >> 5] |= bits << (c & 16);
+                        }
+                    }
+                }
+                tc_fence_before();
+                unsigned und = __ballot_sync(0xffffffffu, undecided);
+                settled += __popc(und);
+                while (und) {
+                    const int i = __ffs(und) - 1;
+                    und &= und - 1;
+                    uint32_t wq[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) wq[q] = __shfl_sync(0xffffffffu, mk[q], i);
+                    const int ri = quarter * 32 + i;
+                    ExactBest best;
+                    best.d = CUDART_INF;
+                    best.k = 0x7FFFFFFF;
+                    // four candidates at a time, in ascending index order: equals keep the lower index
+                    while (wq[0] | wq[1] | wq[2] | wq[3]) {
+                        int k_mine = 0x7FFFFFFF;
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            int k = 0x7FFFFFFF;
+#pragma unroll
+                            for (int q = 3; q >= 0; --q)
+                                if (wq[q]) k = 32 * q + __ffs(wq[q]) - 1;   // (the lowest non-empty word wins: q descends)
+                            if (k != 0x7FFFFFFF) {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    if ((k >> 5) == q) wq[q] &= wq[q] - 1;
+                            }
+                            if ((lane >> 3) == t) k_mine = k;
+                        }
+                        const ExactBest e = best_of_four<CPL>(atile, btile, p.npad, p.K, ri, k_mine, lane);
+                        if (e.d < best.d) best = e;
+                    }
+                    if (lane == i && best.k < p.K && best.d == best.d) lab = best.k;   // (else every distance is NaN)
+                }
+                sh.label[rs][r] = lab;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.lab_full[rs]));
+            }
+            if (lane == 0 && settled) atomicAdd(&sh.queued_pass, settled);
+        } else if (warp >= SM_FIRST_WORKER_WARP) {
+            // ------------------------------------------------------------ worker warps
+            const int w = warp - SM_FIRST_WORKER_WARP;
+            const int col0 = lane * CPL;
+            for (int tile = (int)blockIdx.x; tile < num_tiles; tile += G, ++tcount) {
+                const int rs = (int)(tcount & (uint32_t)(na - 1));
+                const uint32_t rph = (tcount >> p.stage_shift) & 1u;
+                if (!wait_warp(smem_u32(&sh.lab_full[rs]), rph, abort_flag, p.ctl, lane)) break;
+                if (!wait_warp(smem_u32(&sh.a_full[rs]), rph, abort_flag, p.ctl, lane)) break;   // (visibility of the tile)
+                const unsigned char *atile = tiles + (size_t)rs * a_bytes;
+                const int64_t row0 = (int64_t)tile * SM_ROWS;
+                if (w < 4 && p.labels && pass + 1 == p.passes) {
+                    const int64_t row = row0 + w * 32 + lane;
+                    if (row < p.N) p.labels[row] = sh.label[rs][w * 32 + lane];
+                }
+                if (APPLY) {
+                    // rows w, w + 16, ...: four in flight
+#pragma unroll 1
+                    for (int r0 = w; r0 < SM_ROWS; r0 += 4 * SM_WORKERS) {
+                        int l[4];
+                        float y[4][CPL], g[4][CPL], b[4][CPL];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const int r = r0 + t * SM_WORKERS;
+                            l[t] = sh.label[rs][r];
+                            load_cols<CPL>(atile, SM_ROWS, r, col0, y[t]);
+                        }
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const size_t at = (size_t)(l[t] < 0 ? 0 : l[t]) * p.D + col0;
+#pragma unroll
+                            for (int j = 0; j < CPL; ++j) {
+                                g[t][j] = __ldg(p.gamma + at + j);
+                                b[t][j] = __ldg(p.beta + at + j);
+                            }
+                        }
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            if (l[t] < 0) continue;   // beyond the last row (warp-uniform)
+                            float o[CPL];
+#pragma unroll
+                            for (int j = 0; j < CPL; ++j) o[j] = fmaf(g[t][j], y[t][j], b[t][j]);
+                            float *dst = p.out + (size_t)(row0 + r0 + t * SM_WORKERS) * p.D + col0;
+                            if (CPL == 4) __stcs(reinterpret_cast<float4 *>(dst), make_float4(o[0], o[1 % CPL], o[2 % CPL], o[3 % CPL]));
+                            else if (CPL == 2) __stcs(reinterpret_cast<float2 *>(dst), make_float2(o[0], o[1 % CPL]));
+                            else __stcs(dst, o[0]);
+                        }
+                    }
+                } else {
+                    // The rows of this warp's clusters in tile order, so every sum has one fixed order.
+                    // The sums live in shared memory (fp64), each cluster touched by its own warp only.
+                    // A few rows are loaded before they are added.
+#pragma unroll 1
+                    for (int ch = 0; ch < SM_ROWS / 32; ++ch) {
+                        const int lab = sh.label[rs][ch * 32 + lane];
+                        unsigned m = __ballot_sync(0xffffffffu, lab >= 0 && (lab & (SM_WORKERS - 1)) == w);
+                        while (m) {
+                            constexpr int NB = 4;
+                            int k[NB];
+                            float y[NB][CPL];
+#pragma unroll
+                            for (int t = 0; t < NB; ++t) {
+                                k[t] = -1;
+                                if (m) {   // (warp-uniform)
+                                    const int i = __ffs(m) - 1;
+                                    m &= m - 1;
+                                    k[t] = __shfl_sync(0xffffffffu, lab, i);
+                                    load_cols<CPL>(atile, SM_ROWS, ch * 32 + i, col0, y[t]);
+                                }
+                            }
+#pragma unroll
+                            for (int t = 0; t < NB; ++t) {
+                                if (k[t] >= 0) {   // (warp-uniform)
+                                    double *a = sacc + (size_t)k[t] * p.D + col0;
+#pragma unroll
+                                    for (int j = 0; j < CPL; ++j) a[j] += (double)y[t][j];
+                                    if (lane == 0) ++scnt[k[t]];
+                                }
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.a_empty[rs]));
+            }
+            if (!APPLY) {
+                // this CTA's partial sums, and zeros for the next pass (a pass that was cut short leaves
+                // garbage: the status says so)
+                __syncwarp();
+                for (int k = w; k < p.K; k += SM_WORKERS) {
+                    double *a = sacc + (size_t)k * p.D + col0;
+#pragma unroll
+                    for (int j = 0; j < CPL; ++j) {
+                        __stcg(p.part + (size_t)blockIdx.x * (p.K * p.D) + (size_t)k * p.D + col0 + j, a[j]);
+                        a[j] = 0.0;
+                    }
+                    if (lane == 0) {
+                        __stcg(p.part_counts + (size_t)blockIdx.x * (p.K + 1) + k, scnt[k]);
+                        scnt[k] = 0;
+                    }
+                }
+            }
+        }
+
+        __syncthreads();
+        if (APPLY) {
+            // rows that took the exact pass, for the caller's counters (zeroed before the launch)
+            if (tid == 0 && sh.queued_pass) {
+                atomicAdd(reinterpret_cast<unsigned long long *>(&p.ctl->refined_total), (unsigned long long)sh.queued_pass);
+                atomicAdd(reinterpret_cast<unsigned long long *>(&p.ctl->refined_last), (unsigned long long)sh.queued_pass);
+            }
+            break;
+        }
+        const int KD = p.K * p.D;
+        if (tid == 0) {
+            __stcg(p.part_counts + (size_t)blockIdx.x * (p.K + 1) + p.K, sh.queued_pass);
+            sh.queued_pass = 0;
+        }
+        bar_next += (unsigned int)G;
+        if (!grid_barrier(p, bar_next, abort_flag)) { alive = false; break; }
+
+        // ---------------------------------------------------------------- grid-wide combine
+        // One warp per (cluster, column): the CTAs' partials in a fixed order.  The last pass of a
+        // fit leaves the centroids alone (its sums and sizes feed the closed form).
+        const bool update = pass + 1 < p.passes || p.update_last != 0;
+        // (a lane's loads are all issued before the first is used: they are L2 round trips)
+        static_assert(SMALL_MAX_GRID <= 5 * 32, "a lane holds at most five CTAs' partials");
+        for (int e = (int)blockIdx.x * SM_WARPS + warp; e < KD; e += G * SM_WARPS) {
+            const int k = e / p.D;
+            double v[5];
+            int c[5];
+#pragma unroll
+            for (int t = 0; t < 5; ++t) {
+                const int g = lane + 32 * t;
+                v[t] = g < G ? __ldcg(p.part + (size_t)g * KD + e) : 0.0;
+                c[t] = g < G ? __ldcg(p.part_counts + (size_t)g * (p.K + 1) + k) : 0;
+            }
+            double s = v[0];
+            long long n = c[0];
+#pragma unroll
+            for (int t = 1; t < 5; ++t) {
+                if (lane + 32 * t < G) s += v[t];   // (never adds a +0.0 that could turn -0.0 around)
+                n += c[t];
+            }
+            s = warp_sum_f64(s);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+            if (lane == 0) {
+                p.sums[e] = s;
+                if (e == k * p.D) p.counts[k] = n;
+                if (update && n > 0) __stcg(p.C + e, (float)(s / (double)n));
+            }
+        }
+        if (blockIdx.x == 0 && warp == 0) {
+            long long q = 0;
+            for (int g = lane; g < G; g += 32) q += __ldcg(p.part_counts + (size_t)g * (p.K + 1) + p.K);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+            if (lane == 0) {
+                p.ctl->refined_last = q;
+                p.ctl->refined_total += q;
+            }
+        }
+        if (pass + 1 < p.passes) {
+            bar_next += (unsigned int)G;
+            if (!grid_barrier(p, bar_next, abort_flag)) { alive = false; break; }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    if (warp == 1 && lane == 0) {
+        // every MMA this thread issued has completed once this commit arrives
+        tc_commit(smem_u32(&sh.drain));
+        for (int tries = 0; tries < 4000000; ++tries)
+            if (mbar_try_wait(smem_u32(&sh.drain), 0)) break;
+    }
+    if (warp == 0 && lane == 0 && *abort_flag) {
+        // give copies that are still in flight a bounded time to land
+        for (int s = 0; s < na; ++s)
+            for (int tries = 0; tries < 100000; ++tries)
+                if (mbar_try_wait(smem_u32(&sh.a_full[s]), 0) || mbar_try_wait(smem_u32(&sh.a_full[s]), 1)) break;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+}  // namespace
+
+namespace {
+
+struct SmallGeom {
+    int cpl, npad, stages, stage_shift, tmem_cols;
+    size_t smem;
+};
+
+bool small_geometry(int D, int K, bool apply, SmallGeom *g)
+{
+    if (!(D == 32 || D == 64 || D == 128) || K < 1 || K > 128) return false;
+    g->cpl = D / 32;
+    if (!apply && K * D > 4096) return false;   // the fp64 sums take K * D * 8 bytes of shared memory
+    g->npad = (K + 31) / 32 * 32;
+    const int a_bytes = SM_ROWS * D * 4;
+    g->stages = 131072 / a_bytes < SM_MAX_STAGES ? 131072 / a_bytes : SM_MAX_STAGES;   // 4, or 2 at D = 128
+    g->stage_shift = g->stages == 4 ? 2 : 1;
+    int cols = 32;
+    while (cols < g->stages * g->npad) cols <<= 1;
+    g->tmem_cols = cols;
+    g->smem = 1024 + (size_t)g->stages * a_bytes + (size_t)g->npad * D * 4 + (apply ? 0 : (size_t)K * D * 8 + 512) +
+              sizeof(SmallShared);
+    return cols <= 512 && g->smem <= 227 * 1024;
+}
+
+template <bool APPLY, int CPL>
+cudaError_t launch_one(const CUtensorMap &map, const SmallParams &p, int grid, size_t smem, cudaStream_t s)
+{
+    auto kern = small_kernel<APPLY, CPL>;
+    static std::atomic<bool> prepared{false};
+    if (!prepared.load(std::memory_order_acquire)) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        prepared.store(true, std::memory_order_release);
+    }
+    if constexpr (APPLY) {
+        // no CTA waits for another: an ordinary launch, allowed to start early
+        launch_pdl(kern, dim3(grid), dim3(SM_THREADS), smem, s, map, p);
+    } else {
+        // the grid barrier needs every CTA resident
+        int per_sm = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SM_THREADS, smem);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+        void *args[] = {(void *)&map, (void *)&p};
+        e = cudaLaunchCooperativeKernel((const void *)kern, dim3(grid), dim3(SM_THREADS), args, smem, s);
+        if (e != cudaSuccess) return e;
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <bool APPLY>
+cudaError_t dispatch(const SmallGeom &g, const CUtensorMap &map, const SmallParams &p, int grid, cudaStream_t s)
+{
+    if (g.cpl == 1) return launch_one<APPLY, 1>(map, p, grid, g.smem, s);
+    if (g.cpl == 2) return launch_one<APPLY, 2>(map, p, grid, g.smem, s);
+    if (g.cpl == 4) return launch_one<APPLY, 4>(map, p, grid, g.smem, s);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+bool small_fit_supported(int64_t N, int D, int K)
+{
+    SmallGeom g;
+    return N >= SM_ROWS && N < ((int64_t)1 << 31) - SM_ROWS && small_geometry(D, K, false, &g);
+}
+
+bool small_apply_supported(int64_t N, int D, int K)
+{
+    SmallGeom g;
+    return N >= SM_ROWS && N < ((int64_t)1 << 31) - SM_ROWS && small_geometry(D, K, true, &g);
+}
+
+size_t small_part_doubles(int D, int K) { return (size_t)SMALL_MAX_GRID * K * D; }
+size_t small_part_counts(int K) { return (size_t)SMALL_MAX_GRID * (K + 1); }
+
+static int small_grid(int64_t N)
+{
+    int grid = tc_sm_count();
+    if (grid > SMALL_MAX_GRID) grid = SMALL_MAX_GRID;
+    const int64_t tiles = (N + SM_ROWS - 1) / SM_ROWS;
+    if (tiles < grid) grid = (int)tiles;
+    return grid < 1 ? 1 : grid;
+}
+
+// `passes` assignments from the centroids in C; all but the last (and the last too with
+// update_last) replace C by the cluster means.  labels, sums and counts describe the last pass.
+// *bar_count follows the grid barrier's counter (zero after launch_reset_control).
+cudaError_t launch_small_fit(const float *Y, int64_t N, int D, int K, float *C, int passes, bool update_last,
+                             int32_t *labels, double *part, int32_t *part_counts, double *sums, int64_t *counts,
+                             Control *ctl, unsigned int *bar_count, cudaStream_t s)
+{
+    SmallGeom g;
+    if (!small_geometry(D, K, false, &g) || passes < 1) return cudaErrorInvalidValue;
+    CUtensorMap map;
+    if (!tc_make_map(&map, Y, false, N, D, SM_ROWS)) return cudaErrorNotSupported;
+    SmallParams p{};
+    p.Y = Y; p.C = C; p.labels = labels; p.part = part; p.part_counts = part_counts; p.sums = sums; p.counts = counts;
+    p.ctl = ctl; p.bar_base = *bar_count; p.N = N; p.D = D; p.K = K; p.npad = g.npad; p.stages = g.stages; p.stage_shift = g.stage_shift;
+    p.tmem_cols = g.tmem_cols; p.passes = passes; p.update_last = update_last ? 1 : 0;
+    const int grid = small_grid(N);
+    *bar_count += (unsigned int)grid * (unsigned int)(2 * passes - 1);
+    return dispatch<false>(g, map, p, grid, s);
+}
+
+cudaError_t launch_small_apply(const float *Y, int64_t N, int D, int K, const float *C, const float *gamma,
+                               const float *beta, float *out, int32_t *labels, Control *ctl, cudaStream_t s)
+{
+    SmallGeom g;
+    if (!small_geometry(D, K, true, &g)) return cudaErrorInvalidValue;
+    CUtensorMap map;
+    if (!tc_make_map(&map, Y, false, N, D, SM_ROWS)) return cudaErrorNotSupported;
+    SmallParams p{};
+    p.Y = Y; p.C = const_cast<float *>(C); p.labels = labels; p.gamma = gamma; p.beta = beta; p.out = out; p.ctl = ctl;
+    p.N = N; p.D = D; p.K = K; p.npad = g.npad; p.stages = g.stages; p.stage_shift = g.stage_shift; p.tmem_cols = g.tmem_cols; p.passes = 1;
+    return dispatch<true>(g, map, p, small_grid(N), s);
+}
+
+}  // namespace cat

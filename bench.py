@@ -356,6 +356,9 @@ def run_cuda(args):
     apply_kernel = ("apply_h64_kernel (64-row tiles, fp16 operands made in the kernel)"
                     if (form in (0, 64) and K >= B.cat_get_tensor_core_min_k() and K <= 256 and 640 <= D <= 2048
                         and D % 8 == 0 and N_apply >= 4096) else "assign_tc_kernel<affine> / assign_kernel<affine>")
+    if ((B.cat_get_small_problem_kernels() & 1) and D in (32, 64, 128) and B.cat_get_tensor_core_min_k() <= K <= 128
+            and N_apply >= 128):
+        apply_kernel = "small_kernel<inference> (one persistent launch: TF32 scores, in-kernel exact pass, affine from the staged tile)"
     if fp16_rounds:
         # paced by the tensor cores: flop of the distance contraction against the measured dense peak
         roofline_fit = {"bound": "tensor", "kernel": "one Lloyd round of cat_fit (assign_tc_kernel<labels, pair, fp16> + exact "
@@ -380,7 +383,7 @@ def run_cuda(args):
             "fit_s_per_lloyd_iter": lloyd_ms * 1e-3,
             "fit_ms": fit_ms_step, "fit_one_round_ms": fit1_ms, "apply_ms": apply_ms_step,
             "wall_s": t_wall,
-            "roofline": {"bound": "hbm", "kernel": apply_kernel + " (the one kernel of cat_apply besides the exact pass)",
+            "roofline": {"bound": "hbm", "kernel": apply_kernel + ("" if apply_kernel.startswith("small_kernel") else " (the one kernel of cat_apply besides the exact pass)"),
                          "achieved": apply_gbs, "peak": peak, "unit": "GB/s", "frac": apply_gbs / peak,
                          "peak_source": peak_src, "traffic": traffic},
             "roofline_fit": roofline_fit,

@@ -9,10 +9,12 @@
 //   warp 0      TMA producer: a row tile (128 x D fp32, 128-byte swizzle) per ring stage
 //   warp 1      issues the TF32 tcgen05.mma of the tile against all centroids (accumulator in
 //               TMEM, one buffer per ring stage)
-//   warps 4-11  score warps, two sets of four that take alternate tiles: read the scores from
-//               TMEM, keep the four smallest keys per row and take the certainty test; the rows that
-//               fail it are settled at once by the warp together (fp64 direct form over the listed
-//               candidates, or over all K), so the labels that leave these warps are final
+//   warps 4-11  score warps, two sets of four that take alternate tiles: a thread owns a row, reads
+//               its scores from TMEM, keeps the four smallest keys and takes the certainty test; a
+//               row that fails it is settled at once by its own thread (fp64 direct form over the
+//               centroids whose key lies within the error bound of the best -- found by a second
+//               read of the scores when there may be more than four), so the labels that leave
+//               these warps are final
 //   warps 12-27 worker warps: either add the tile's rows to per-cluster fp64 sums in shared memory
 //               (warp w owns the clusters k = w mod 16, a lane owns D / 32 columns), or write
 //               gamma_l * y + beta_l.
@@ -25,10 +27,10 @@
 // The launch is cooperative (all CTAs resident), and every wait -- on an mbarrier or on the grid
 // barrier -- gives up after a time limit, raises the device status and lets the kernel return.
 //
-// Measured on 200 704 x 64 rows, K = 64: inference 74 us against 85 us for the general path; a
-// Lloyd round 81 us against 57 us (per-tile handoffs between the warp roles, the exact pass on
-// about 15 % of the rows -- TF32 scores -- and two grid barriers a round cost more than the launches
-// they replace), so fitting takes this kernel only on request.
+// Measured on 200 704 x 64 rows, K = 64: inference 56 us against 86 us for the general path; a
+// Lloyd round 60 us against 57 us (the exact pass on about 15 % of the rows -- TF32 scores --, the
+// per-tile handoffs between the warp roles and two grid barriers a round cost what the launches
+// they replace cost), so fitting takes this kernel only on request.
 #include "cat_tc.cuh"
 
 namespace cat {
@@ -37,23 +39,20 @@ namespace {
 constexpr int SM_ROWS = 128;                 // rows per tile
 constexpr int SM_MAX_STAGES = 4;
 constexpr unsigned SM_POLL_SLEEP_NS = 100;
+constexpr int SM_PART_PAD = 48;              // doubles between the CTAs' planes of partial sums (no power-of-two stride)
 constexpr int SM_FIRST_SCORE_WARP = 4;
 constexpr int SM_FIRST_WORKER_WARP = 12;     // warps 4-11: two sets of four score warps
 constexpr int SM_WORKERS = 16;
 constexpr int SM_WARPS = SM_FIRST_WORKER_WARP + SM_WORKERS;   // 28
 constexpr int SM_THREADS = 32 * SM_WARPS;                     // 896
 
-struct ExactBest {
-    double d;
-    int k;
-};
-
 struct SmallParams {
     const float *Y;          // [N, D]
     float *C;                // [K, D] centroids, updated in place by a round
     int32_t *labels;         // [N] labels of the last pass (written in that pass only; may be null)
     double *part;            // [grid, K * D] partial sums of a CTA
-    int32_t *part_counts;    // [grid, K + 1] partial sizes of a CTA, then its count of queued rows
+    int32_t *part_counts;    // [2, K + 1] cluster sizes, then the count of queued rows, of the even and odd passes
+                             // (both planes zero at launch)
     double *sums;            // [K * D] per-cluster sums of the last pass
     int64_t *counts;         // [K]
     const float *gamma;      // inference only
@@ -183,42 +182,42 @@ __device__ __forceinline__ double warp_sum_f64(double v)
     return v;
 }
 
-// Exact choice among up to four centroids for one row, by one warp: lanes 8g .. 8g + 7 form
-// ||y - c||^2 in fp64 (direct form) for candidate g -- a lane takes D / 8 consecutive columns in
-// order, then a fixed three-step tree inside the group -- and the four groups are compared:
-// the smallest distance wins, the lowest index among equals.  A candidate index >= K is unused
-// (distance +inf).  The result is the same in every lane.
-template <int CPL>
-__device__ __forceinline__ ExactBest best_of_four(const unsigned char *atile, const unsigned char *btile, int npad,
-                                                  int K, int r, int k_mine, int lane)
+// index of the lowest set bit of a 128-bit mask held in four words, which it clears; -1 if none
+__device__ __forceinline__ int pop_lowest(uint32_t &m0, uint32_t &m1, uint32_t &m2, uint32_t &m3)
 {
-    const int sub = lane & 7;
-    const bool valid = k_mine < K;
-    const int kc = valid ? k_mine : 0;
-    double s = 0.0;
-#pragma unroll
-    for (int i = 0; i < CPL; ++i) {
-        const int col = 4 * (sub * CPL + i);
-        const float4 y = *reinterpret_cast<const float4 *>(atile + swz(SM_ROWS, r, col));
-        const float4 c = *reinterpret_cast<const float4 *>(btile + swz(npad, kc, col));
+    int k = -1;
+    if (m0) { k = __ffs(m0) - 1; m0 &= m0 - 1; }
+    else if (m1) { k = 31 + __ffs(m1); m1 &= m1 - 1; }
+    else if (m2) { k = 63 + __ffs(m2); m2 &= m2 - 1; }
+    else if (m3) { k = 95 + __ffs(m3); m3 &= m3 - 1; }
+    return k;
+}
+
+// ||y - c_a||^2 and ||y - c_b||^2 in fp64 (direct form) for row r of the staged tile, by one thread:
+// columns in order, even and odd columns in two partial sums each.
+template <int CPL>
+__device__ __forceinline__ void exact_pair(const unsigned char *atile, const unsigned char *btile, int npad, int r,
+                                           int ka, int kb, double &da, double &db)
+{
+    double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;
+#pragma unroll 4
+    for (int c4 = 0; c4 < 8 * CPL; ++c4) {
+        const float4 y = *reinterpret_cast<const float4 *>(atile + swz(SM_ROWS, r, c4 * 4));
+        const float4 ca = *reinterpret_cast<const float4 *>(btile + swz(npad, ka, c4 * 4));
+        const float4 cb = *reinterpret_cast<const float4 *>(btile + swz(npad, kb, c4 * 4));
+        const double y0 = (double)y.x, y1 = (double)y.y, y2 = (double)y.z, y3 = (double)y.w;
         double d;
-        d = (double)y.x - (double)c.x; s = fma(d, d, s);
-        d = (double)y.y - (double)c.y; s = fma(d, d, s);
-        d = (double)y.z - (double)c.z; s = fma(d, d, s);
-        d = (double)y.w - (double)c.w; s = fma(d, d, s);
+        d = y0 - (double)ca.x; a0 = fma(d, d, a0);
+        d = y1 - (double)ca.y; a1 = fma(d, d, a1);
+        d = y2 - (double)ca.z; a0 = fma(d, d, a0);
+        d = y3 - (double)ca.w; a1 = fma(d, d, a1);
+        d = y0 - (double)cb.x; b0 = fma(d, d, b0);
+        d = y1 - (double)cb.y; b1 = fma(d, d, b1);
+        d = y2 - (double)cb.z; b0 = fma(d, d, b0);
+        d = y3 - (double)cb.w; b1 = fma(d, d, b1);
     }
-#pragma unroll
-    for (int o = 1; o < 8; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    ExactBest b;
-    b.d = valid ? s : CUDART_INF;
-    b.k = valid ? k_mine : 0x7FFFFFFF;
-#pragma unroll
-    for (int o = 8; o < 32; o <<= 1) {
-        const double d2 = __shfl_xor_sync(0xffffffffu, b.d, o);
-        const int k2 = __shfl_xor_sync(0xffffffffu, b.k, o);
-        if (d2 < b.d || (d2 == b.d && k2 < b.k) || (b.d != b.d && d2 == d2)) { b.d = d2; b.k = k2; }
-    }
-    return b;
+    da = a0 + a1;
+    db = b0 + b1;
 }
 
 // APPLY: inference (one pass, no sums, no grid barrier).  CPL = D / 32 columns per lane,
@@ -402,7 +401,7 @@ small_kernel(const __grid_constant__ CUtensorMap mapA, SmallParams p)
                 // Candidates of an undecided row, one bit per centroid: those whose key lies within the
                 // limit of the best.  When the fourth smallest key is still inside the limit the row's
                 // scores are read once more from TMEM to find them all.
-                uint32_t mk[4] = {0u, 0u, 0u, 0u};
+                uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
                 bool undecided = false, wide = false;
                 float lim = 0.f;
                 if (row < p.N) {
@@ -417,9 +416,11 @@ small_kernel(const __grid_constant__ CUtensorMap mapA, SmallParams p)
                             for (int t = 0; t < 4; ++t) {
                                 const int k = key_index(bk[t]);
                                 if (t < p.K && !((bk[t] - b1) > lim)) {
-#pragma unroll
-                                    for (int q = 0; q < 4; ++q)
-                                        if ((k >> 5) == q) mk[q] |= 1u << (k & 31);
+                                    const uint32_t bit = 1u << (k & 31);
+                                    if (k < 32) m0 |= bit;
+                                    else if (k < 64) m1 |= bit;
+                                    else if (k < 96) m2 |= bit;
+                                    else if (k < 128) m3 |= bit;
                                 }
                             }
                         }
@@ -438,43 +439,34 @@ small_kernel(const __grid_constant__ CUtensorMap mapA, SmallParams p)
                                 const float key = make_key(fmaf(-2.f, __uint_as_float(ra[j]), sh.cn[c + j]), c + j);
                                 if (c + j < p.K && !((key - b1) > lim)) bits |= 1u << j;
                             }
-                            if (wide) mk[c >> 5] |= bits << (c & 16);
+                            if (wide) {   // (c is a constant here: one of these lines remains)
+                                if (c < 32) m0 |= bits << (c & 16);
+                                else if (c < 64) m1 |= bits << (c & 16);
+                                else if (c < 96) m2 |= bits << (c & 16);
+                                else m3 |= bits << (c & 16);
+                            }
                         }
                     }
                 }
                 tc_fence_before();
-                unsigned und = __ballot_sync(0xffffffffu, undecided);
-                settled += __popc(und);
-                while (und) {
-                    const int i = __ffs(und) - 1;
-                    und &= und - 1;
-                    uint32_t wq[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) wq[q] = __shfl_sync(0xffffffffu, mk[q], i);
-                    const int ri = quarter * 32 + i;
-                    ExactBest best;
-                    best.d = CUDART_INF;
-                    best.k = 0x7FFFFFFF;
-                    // four candidates at a time, in ascending index order: equals keep the lower index
-                    while (wq[0] | wq[1] | wq[2] | wq[3]) {
-                        int k_mine = 0x7FFFFFFF;
-#pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            int k = 0x7FFFFFFF;
-#pragma unroll
-                            for (int q = 3; q >= 0; --q)
-                                if (wq[q]) k = 32 * q + __ffs(wq[q]) - 1;   // (the lowest non-empty word wins: q descends)
-                            if (k != 0x7FFFFFFF) {
-#pragma unroll
-                                for (int q = 0; q < 4; ++q)
-                                    if ((k >> 5) == q) wq[q] &= wq[q] - 1;
-                            }
-                            if ((lane >> 3) == t) k_mine = k;
+                // The exact pass, inside the thread that owns the row (all undecided rows of the warp at
+                // once): ||y - c||^2 in fp64 (direct form) for the row's candidates in ascending index
+                // order, two at a time; the smallest wins, the lowest index among equals.
+                settled += __popc(__ballot_sync(0xffffffffu, undecided));
+                {
+                    double best = CUDART_INF;
+                    int bk = -1;
+                    while (__any_sync(0xffffffffu, (m0 | m1 | m2 | m3) != 0u)) {
+                        const int ka = pop_lowest(m0, m1, m2, m3), kb = pop_lowest(m0, m1, m2, m3);
+                        if (ka >= 0) {
+                            double da, db;
+                            const int kaa = ka < p.K ? ka : 0, kbb = (kb >= 0 && kb < p.K) ? kb : 0;
+                            exact_pair<CPL>(atile, btile, p.npad, r, kaa, kbb, da, db);
+                            if (ka < p.K && da < best) { best = da; bk = ka; }
+                            if (kb >= 0 && kb < p.K && db < best) { best = db; bk = kb; }
                         }
-                        const ExactBest e = best_of_four<CPL>(atile, btile, p.npad, p.K, ri, k_mine, lane);
-                        if (e.d < best.d) best = e;
                     }
-                    if (lane == i && best.k < p.K && best.d == best.d) lab = best.k;   // (else every distance is NaN)
+                    if (bk >= 0) lab = bk;   // (else every distance is NaN: the fast label stands)
                 }
                 sh.label[rs][r] = lab;
                 __syncwarp();
@@ -574,11 +566,12 @@ small_kernel(const __grid_constant__ CUtensorMap mapA, SmallParams p)
                     double *a = sacc + (size_t)k * p.D + col0;
 #pragma unroll
                     for (int j = 0; j < CPL; ++j) {
-                        __stcg(p.part + (size_t)blockIdx.x * (p.K * p.D) + (size_t)k * p.D + col0 + j, a[j]);
+                        __stcg(p.part + (size_t)blockIdx.x * (p.K * p.D + SM_PART_PAD) + (size_t)k * p.D + col0 + j, a[j]);
                         a[j] = 0.0;
                     }
                     if (lane == 0) {
-                        __stcg(p.part_counts + (size_t)blockIdx.x * (p.K + 1) + k, scnt[k]);
+                        // (integer sums do not depend on the order: one atomic a cluster and CTA)
+                        if (scnt[k]) atomicAdd(p.part_counts + (size_t)(pass & 1) * (p.K + 1) + k, scnt[k]);
                         scnt[k] = 0;
                     }
                 }
@@ -596,54 +589,51 @@ small_kernel(const __grid_constant__ CUtensorMap mapA, SmallParams p)
         }
         const int KD = p.K * p.D;
         if (tid == 0) {
-            __stcg(p.part_counts + (size_t)blockIdx.x * (p.K + 1) + p.K, sh.queued_pass);
+            if (sh.queued_pass) atomicAdd(p.part_counts + (size_t)(pass & 1) * (p.K + 1) + p.K, sh.queued_pass);
             sh.queued_pass = 0;
         }
         bar_next += (unsigned int)G;
         if (!grid_barrier(p, bar_next, abort_flag)) { alive = false; break; }
 
         // ---------------------------------------------------------------- grid-wide combine
-        // One warp per (cluster, column): the CTAs' partials in a fixed order.  The last pass of a
-        // fit leaves the centroids alone (its sums and sizes feed the closed form).
+        // One warp per four neighbouring columns of a cluster: lane (g8, c) takes column c of the CTAs
+        // g8, g8 + 8, ... in that order, so that the four lanes of a CTA read one 32-byte sector
+        // together, and a fixed three-step tree adds the eight partial sums.  The last pass of a fit
+        // leaves the centroids alone (its sums and sizes feed the closed form).
         const bool update = pass + 1 < p.passes || p.update_last != 0;
-        // (a lane's loads are all issued before the first is used: they are L2 round trips)
-        static_assert(SMALL_MAX_GRID <= 5 * 32, "a lane holds at most five CTAs' partials");
-        for (int e = (int)blockIdx.x * SM_WARPS + warp; e < KD; e += G * SM_WARPS) {
+        const int32_t *kcount = p.part_counts + (size_t)(pass & 1) * (p.K + 1);
+        static_assert(SMALL_MAX_GRID <= 8 * 20, "a lane holds at most twenty CTAs' partials");
+        for (int e4 = (int)blockIdx.x * SM_WARPS + warp; e4 < (KD >> 2); e4 += G * SM_WARPS) {
+            const int e = 4 * e4 + (lane & 3);
             const int k = e / p.D;
-            double v[5];
-            int c[5];
+            // (a lane's loads are all issued before the first is used: they are L2 round trips)
+            double v[20];
 #pragma unroll
-            for (int t = 0; t < 5; ++t) {
-                const int g = lane + 32 * t;
-                v[t] = g < G ? __ldcg(p.part + (size_t)g * KD + e) : 0.0;
-                c[t] = g < G ? __ldcg(p.part_counts + (size_t)g * (p.K + 1) + k) : 0;
+            for (int t = 0; t < 20; ++t) {
+                const int g = (lane >> 2) + 8 * t;
+                v[t] = g < G ? __ldcg(p.part + (size_t)g * (KD + SM_PART_PAD) + e) : 0.0;
             }
+            const long long n = __ldcg(kcount + k);
             double s = v[0];
-            long long n = c[0];
 #pragma unroll
-            for (int t = 1; t < 5; ++t) {
-                if (lane + 32 * t < G) s += v[t];   // (never adds a +0.0 that could turn -0.0 around)
-                n += c[t];
-            }
-            s = warp_sum_f64(s);
+            for (int t = 1; t < 20; ++t)
+                if ((lane >> 2) + 8 * t < G) s += v[t];   // (never adds a +0.0 that could turn -0.0 around)
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
-            if (lane == 0) {
+            for (int o = 4; o < 32; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane < 4) {
                 p.sums[e] = s;
                 if (e == k * p.D) p.counts[k] = n;
                 if (update && n > 0) __stcg(p.C + e, (float)(s / (double)n));
             }
         }
-        if (blockIdx.x == 0 && warp == 0) {
-            long long q = 0;
-            for (int g = lane; g < G; g += 32) q += __ldcg(p.part_counts + (size_t)g * (p.K + 1) + p.K);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-            if (lane == 0) {
-                p.ctl->refined_last = q;
-                p.ctl->refined_total += q;
-            }
+        if (blockIdx.x == 0 && warp == 0 && lane == 0) {
+            const long long q = __ldcg(kcount + p.K);
+            p.ctl->refined_last = q;
+            p.ctl->refined_total += q;
         }
+        // the other plane of counts is the next pass's: nobody reads or adds to it before the barrier below
+        if (blockIdx.x == 0)
+            for (int i = tid; i <= p.K; i += SM_THREADS) p.part_counts[(size_t)((pass + 1) & 1) * (p.K + 1) + i] = 0;
         if (pass + 1 < p.passes) {
             bar_next += (unsigned int)G;
             if (!grid_barrier(p, bar_next, abort_flag)) { alive = false; break; }
@@ -748,8 +738,8 @@ bool small_apply_supported(int64_t N, int D, int K)
     return N >= SM_ROWS && N < ((int64_t)1 << 31) - SM_ROWS && small_geometry(D, K, true, &g);
 }
 
-size_t small_part_doubles(int D, int K) { return (size_t)SMALL_MAX_GRID * K * D; }
-size_t small_part_counts(int K) { return (size_t)SMALL_MAX_GRID * (K + 1); }
+size_t small_part_doubles(int D, int K) { return (size_t)SMALL_MAX_GRID * ((size_t)K * D + SM_PART_PAD); }
+size_t small_part_counts(int K) { return 2 * ((size_t)K + 1); }
 
 static int small_grid(int64_t N)
 {
@@ -775,6 +765,8 @@ cudaError_t launch_small_fit(const float *Y, int64_t N, int D, int K, float *C, 
     p.Y = Y; p.C = C; p.labels = labels; p.part = part; p.part_counts = part_counts; p.sums = sums; p.counts = counts;
     p.ctl = ctl; p.bar_base = *bar_count; p.N = N; p.D = D; p.K = K; p.npad = g.npad; p.stages = g.stages; p.stage_shift = g.stage_shift;
     p.tmem_cols = g.tmem_cols; p.passes = passes; p.update_last = update_last ? 1 : 0;
+    cudaError_t e0 = cudaMemsetAsync(part_counts, 0, small_part_counts(K) * sizeof(int32_t), s);
+    if (e0 != cudaSuccess) return e0;
     const int grid = small_grid(N);
     *bar_count += (unsigned int)grid * (unsigned int)(2 * passes - 1);
     return dispatch<false>(g, map, p, grid, s);

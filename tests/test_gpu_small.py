@@ -39,7 +39,7 @@ def _data(seed, n, d, spread=3.0):
 SHAPES = [(1000, 32, 40), (5000, 128, 32), (333, 64, 33), (128, 64, 64), (20001, 64, 64), (3000, 32, 128)]
 
 
-@pytest.mark.parametrize("n,d,k", SHAPES)
+@pytest.mark.parametrize("n,d,k", SHAPES + [(2000, 128, 128), (4097, 64, 128), (129, 32, 32)])
 def test_inference_matches_the_oracle(n, d, k, small_mask):
     Yq, _ = _data(n + d + k, n, d)
     rng = np.random.default_rng(7)
@@ -156,3 +156,31 @@ def test_many_candidates_and_exact_ties(small_mask):
     Cf, _, _, labels = B.cat_fit(dev(Yq), dev(Yq), k, 1, init_centroids=dev(C))
     lab1, best1, second1 = O.assign(Yq, host(Cf))
     labels_match(host(labels), lab1, best1, second1, "fit labels, bunched centroids")
+
+
+def test_fit_without_rounds_is_the_assignment_to_the_first_rows(small_mask):
+    """iters = 0: one pass of the persistent kernel that leaves the centroids alone; its sums and
+    sizes still feed the closed form."""
+    n, d, k = 3000, 64, 48
+    Yq, Yfp = _data(99, n, d)
+    B.cat_set_small_problem_kernels(3)
+    C, G, Bt, labels = B.cat_fit(dev(Yq), dev(Yfp), k, 0)
+    assert np.array_equal(host(C), Yq[:k])
+    lab, best, second = O.assign(Yq, Yq[:k])
+    labels_match(host(labels), lab, best, second, "labels of a fit without rounds")
+    g_want, b_want = O.solve_gamma_beta(Yq, Yfp, host(labels), k)
+    close(host(G), g_want, "gamma")
+    close(host(Bt), b_want, "beta")
+
+
+def test_shapes_outside_the_small_kernels_take_the_general_path(small_mask):
+    """K * D above 4096 (fitting) or a D that is not 32, 64 or 128: same results, other kernels."""
+    B.cat_set_small_problem_kernels(3)
+    for n, d, k in [(2000, 128, 64), (1500, 96, 40)]:
+        Yq, Yfp = _data(n + d, n, d)
+        C, G, Bt, labels = B.cat_fit(dev(Yq), dev(Yfp), k, 3)
+        lab, best, second = O.assign(Yq, host(C))
+        labels_match(host(labels), lab, best, second, f"labels, D = {d}, K = {k}")
+        out = B.cat_apply(dev(Yq), C, G, Bt)
+        want = O.affine_with_labels(Yq, host(labels), host(G), host(Bt))
+        close(host(out), want, f"outputs, D = {d}, K = {k}")

@@ -359,7 +359,15 @@ def run_cuda(args):
     if ((B.cat_get_small_problem_kernels() & 1) and D in (32, 64, 128) and B.cat_get_tensor_core_min_k() <= K <= 128
             and N_apply >= 128):
         apply_kernel = "small_kernel<inference> (one persistent launch: TF32 scores, in-kernel exact pass, affine from the staged tile)"
-    if fp16_rounds:
+    small_fit = ((B.cat_get_small_problem_kernels() & 2) and D in (32, 64, 128) and K * D <= 4096
+                 and B.cat_get_tensor_core_min_k() <= K <= 128 and N_fit >= 128)
+    if small_fit:
+        # all rounds in one persistent launch: a round reads the fp32 rows once (TF32 scores from the staged tile)
+        roofline_fit = {"bound": "hbm", "kernel": "one Lloyd round inside small_kernel<fit> (one cooperative launch for the "
+                        "whole fit: TF32 scores, in-kernel exact pass, fp64 sums in shared memory, ordered grid-wide combine)",
+                        "achieved": lloyd_alg_gbs, "peak": peak, "unit": "GB/s", "frac": lloyd_alg_gbs / peak,
+                        "peak_source": peak_src, "tflops": lloyd_tflops}
+    elif fp16_rounds:
         # paced by the tensor cores: flop of the distance contraction against the measured dense peak
         roofline_fit = {"bound": "tensor", "kernel": "one Lloyd round of cat_fit (assign_tc_kernel<labels, pair, fp16> + exact "
                         "pass + changed-row sums + centroid update)", "achieved": lloyd_tflops, "peak": peak_tf,

@@ -401,11 +401,12 @@ int32_t cat_get_tensor_core_min_k(void);
  * rows; K >= the tensor-core threshold above) have persistent single-launch kernels: scores on the
  * tensor cores, undecided rows settled in fp64 inside the kernel, and for fitting the per-cluster
  * sums kept on chip and combined across the grid in a fixed order, all rounds in one launch.
- * mask bit 0: the whole of cat_apply (Algorithm 2) runs that way (default: on -- it is the faster
- * form where it applies).  mask bit 1: so do the K-Means rounds of cat_fit / cat_fit_from
- * (Algorithm 1, step 2; calls without per-round diagnostics) (default: off -- measured slower than
- * the general multi-launch path; kept as a tested alternative).  Same labels either way; sums that
- * agree to fp64 rounding.  A PROCESS-WIDE tuning and test hook like the one above. */
+ * mask bit 0: the whole of cat_apply (Algorithm 2) runs that way.  mask bit 1: so do the K-Means
+ * rounds and the final assignment of cat_fit / cat_fit_from (Algorithm 1, step 2; calls without
+ * per-round diagnostics).  Default 3: both are the faster form where they apply.  Clearing a bit
+ * sends these shapes down the general multi-launch path instead: same labels (rows on a bisector
+ * apart, when a centroid differs in its last bit); sums that agree to fp64 rounding.  A PROCESS-WIDE
+ * tuning and test hook like the one above. */
 void cat_set_small_problem_kernels(int32_t mask);
 int32_t cat_get_small_problem_kernels(void);
 

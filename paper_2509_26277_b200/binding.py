@@ -560,7 +560,7 @@ def cat_get_tensor_core_min_k() -> int:
 
 def cat_set_small_problem_kernels(mask: int) -> None:
     """Process-wide switch of the persistent single-launch kernels for small shapes:
-    bit 0 = inference (default on), bit 1 = the K-Means rounds of a fit (default off)."""
+    bit 0 = inference, bit 1 = the K-Means rounds of a fit (default 3: both on)."""
     lib().cat_set_small_problem_kernels(int(mask))
 
 

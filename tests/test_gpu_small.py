@@ -1,6 +1,5 @@
 """The persistent single-launch kernels for small shapes (D in {32, 64, 128}, K <= 128), through
-the C ABI, against the CPU oracle: inference (on by default where the shape allows it) and the
-K-Means rounds of a fit (on request), including rows that need the exact pass over two, four and
+the C ABI, against the CPU oracle: inference and the K-Means rounds of a fit, including rows that need the exact pass over two, four and
 all K centroids, a ragged last tile, exact ties and run-to-run repeatability."""
 import numpy as np
 import pytest

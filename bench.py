@@ -198,6 +198,10 @@ def run_cuda(args):
     from paper_2509_26277_b200 import binding as B
     from paper_2509_26277_b200 import sharded
 
+    if args.tc_min_k is not None:
+        B.cat_set_tensor_core_min_k(args.tc_min_k)
+    if args.small_kernels is not None:
+        B.cat_set_small_problem_kernels(args.small_kernels)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -322,7 +326,7 @@ def run_cuda(args):
         lloyd_ms = max(fit_ms_step - fit1_ms, 0.0) / (iters - 1)
     else:
         lloyd_ms = fit_ms_step / (iters + 1)
-    # What a round moves and computes.  With K >= 32 and D % 8 == 0 the assignment reads the fp16 copy of
+    # What a round moves and computes.  With K at or above the tensor threshold and D % 8 == 0 the assignment reads the fp16 copy of
     # the rows (N D 2 bytes, plus labels) and is paced by the tensor cores (2 N K D flop); otherwise it
     # reads the fp32 rows.  The algorithmic figure (one fp32 read of Yq per round) is reported beside it.
     fp16_rounds = (K >= B.cat_get_tensor_core_min_k() and D % 8 == 0 and K <= 256 and B.cat_tensor_path_available())
@@ -386,7 +390,8 @@ def run_cuda(args):
             "config": {"workload": f"config {args.config} ({sp['name']})", "N_fit": N_fit, "N_apply": N_apply,
                        "D": D, "K": K, "iters": iters, "rows_scale": args.rows_scale,
                        "l2": "inputs larger than L2" if N_apply * D * 4 > 126e6 else "L2-resident inputs",
-                       "parallelism": f"rows x{world}"},
+                       "parallelism": f"rows x{world}", "tensor_core_min_k": B.cat_get_tensor_core_min_k(),
+                       "small_kernels": B.cat_get_small_problem_kernels()},
             "apply_rows_per_s": N_apply * world / (apply_ms_step * 1e-3),
             "fit_s_per_lloyd_iter": lloyd_ms * 1e-3,
             "fit_ms": fit_ms_step, "fit_one_round_ms": fit1_ms, "apply_ms": apply_ms_step,
@@ -495,6 +500,10 @@ def main():
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--rows-scale", type=float, default=1.0, dest="rows_scale")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--tensor-core-min-k", type=int, default=None, dest="tc_min_k",
+                    help="kernel selection: tensor-core scores for K >= this (library default 32)")
+    ap.add_argument("--small-kernels", type=int, default=None, dest="small_kernels",
+                    help="kernel selection: mask of the persistent small-shape kernels (library default 3)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--check", action="store_true",

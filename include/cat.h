@@ -389,8 +389,10 @@ cat_status_t cat_selftest_wait_timeout(void *workspace, size_t workspace_bytes, 
 /* Kernel selection for the distance contraction.  With K >= min_k (and D % 4 == 0,
  * K <= 256) the scores are formed on the tensor cores (tcgen05, TF32 or fp16 operands, fp32
  * accumulation); below it on the fp32 pipes.  Either way undecided rows are settled in
- * fp64, so the labels are the same.  Default 32: for smaller K the contraction is not
- * compute-limited.
+ * fp64, so the labels are the same.  Default 8: measured at K = 8, 16 and 32 (rows of 1000
+ * columns) a Lloyd round takes half the time on the tensor path and so does inference, except
+ * where low-precision scores leave most rows undecided (unimodal data, K = 32: there the fp32
+ * pipes are a quarter faster for inference).
  * This and cat_set_apply_column_split are PROCESS-WIDE tuning and test hooks: they change
  * which kernel every later call of every thread launches (never the results), and they are
  * not meant to be flipped while other threads are inside the library. */

@@ -103,7 +103,7 @@ static cat_status_t check_shape(int64_t N, int32_t D, int32_t K, bool need_n_ge_
         if (!cuda_ok((expr))) return CAT_ERR_CUDA;      \
     } while (0)
 
-static std::atomic<int> g_tc_min_k{32};
+static std::atomic<int> g_tc_min_k{8};
 static std::atomic<int> g_small_kernels{3};   // bit 0: inference, bit 1: the K-Means rounds of a fit
 
 static bool use_tensor_path(int64_t N, int D, int K)

@@ -96,11 +96,12 @@ def test_whole_fit_against_the_oracle(small_mask):
     Yfp = (means[which] + rng.normal(size=(n, d))).astype(np.float32)
     Yq = (Yfp + 0.05 * rng.normal(size=(n, d))).astype(np.float32)
     B.cat_set_small_problem_kernels(3)
+    old = B.cat_get_tensor_core_min_k()
     B.cat_set_tensor_core_min_k(1)
     try:
         C, G, Bt, labels = B.cat_fit(dev(Yq), dev(Yfp), k, 6)
     finally:
-        B.cat_set_tensor_core_min_k(32)
+        B.cat_set_tensor_core_min_k(old)
     ora = O.fit(Yq, Yfp, k, 6)
     assert np.array_equal(host(labels), ora.labels)
     close(host(C), ora.centroids, "centroids")
